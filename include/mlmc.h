@@ -1,0 +1,136 @@
+/*
+ * mlmc.h: C ABI of the MLMC gradient-compression hot path (CUDA, sm_100a).
+ *
+ * The library turns a biased multilevel compressor C^l (Def. 3.1) into the unbiased MLMC estimate
+ *     g~ = g^0 + (1/p^l)(C^l(g) - C^{l-1}(g)),   g^0 = 0,   l ~ p            (Eq. 5; Alg. 2 / Alg. 3)
+ * for each of M workers, emits each worker's message, and averages the M messages on the server
+ * side (Alg. 2, "Server aggregates").  Two compressor families are covered: Top-k with a level
+ * schedule k_0 <= ... <= k_{L-1} = d (Sec. 3.2) and fixed-point bit truncation with a bit schedule
+ * b_0 < ... < b_{L-1} <= 23 (Sec. 3.1).  Probabilities are either given (Alg. 2) or adaptive,
+ * p^l proportional to ||C^l(g) - C^{l-1}(g)||_2 per worker per step (Lemma 3.4, Alg. 3).
+ *
+ * Conventions
+ *  - Levels are indexed l = 0..L-1 here; this is the paper's l = 1..L.  k_{-1} = 0, b_{-1} = 0.
+ *  - Pointers are DEVICE pointers unless marked "host".  The caller owns every buffer; the library
+ *    only owns the scratch workspace inside mlmc_ctx.
+ *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default
+ *    stream).  Nothing synchronises except mlmc_create, mlmc_destroy, mlmc_get_status and mlmc_read_u.
+ *  - The int return value reports host-side checks made before any launch (arguments, schedule,
+ *    probabilities).  Conditions found on the device (message capacity, non-finite input, a bounded
+ *    wait that gave up) are written to a sticky status word read by mlmc_get_status; the affected
+ *    worker's message then has count = 0 (Top-k) or level = -1.  Nothing traps or spins unbounded.
+ *  - g is [M][ld] with row stride ld >= d elements, worker m in row m; g must be 16-byte aligned and,
+ *    when M > 1, ld * sizeof(element) must be a multiple of 16.  d < 2^32.  g is never written.
+ *  - Total order for Top-k: |g_i| descending, equal magnitudes by ascending index i.
+ *  - One uniform per (seed, step, worker) drives the level draw: three chained SplitMix64 output
+ *    rounds, u = (h >> 11) * 2^-53; cdf accumulated in ascending l in fp64, the cdf of the last level
+ *    with p > 0 set to 1, l* = min{ l : u < cdf_l }.
+ *  - One mlmc_ctx serves one stream at a time.
+ */
+#ifndef MLMC_H
+#define MLMC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mlmc_ctx mlmc_ctx;
+
+typedef enum { MLMC_F32 = 0, MLMC_BF16 = 1 } mlmc_dtype;
+typedef enum { MLMC_TOPK = 0, MLMC_BITWISE = 1 } mlmc_kind;
+
+typedef enum {
+    MLMC_OK = 0,
+    MLMC_ERR_ARG = -1,       /* null pointer, size out of range, misaligned g, limits of the ctx exceeded */
+    MLMC_ERR_SCHEDULE = -2,  /* k not nondecreasing or k_{L-1} != d;  b not increasing or b_{L-1} > 23 */
+    MLMC_ERR_PROB = -3,      /* some p_l <= 0 or sum p != 1 (Lemma 3.2 needs non-zero probabilities) */
+    MLMC_ERR_CAPACITY = -4,  /* device: a Top-k message does not fit out->capacity / planes exceed w_max */
+    MLMC_ERR_NONFINITE = -5, /* device: NaN or Inf in g */
+    MLMC_ERR_TIMEOUT = -6,   /* device: a bounded wait between thread blocks gave up */
+    MLMC_ERR_CUDA = -7,      /* a CUDA runtime call failed */
+    MLMC_ERR_NOMEM = -8,     /* workspace allocation failed */
+    MLMC_ERR_INTERNAL = -9   /* device: a self-check failed (emitted count differs from k_l - k_{l-1}) */
+} mlmc_status;
+
+#define MLMC_MAX_LEVELS 32
+
+/* Top-k message batch (Sec. 3.2: the residual C^l - C^{l-1} is the band of ranks (k_{l-1}, k_l]).
+ * Structure of arrays in device memory.  Worker m owns idx[m*capacity ..] and val[m*capacity ..]. */
+typedef struct {
+    uint32_t* idx;     /* [M][capacity] coordinates of the band, ascending                         */
+    float*    val;     /* [M][capacity] g_i / p_l                                                  */
+    int64_t*  count;   /* [M] entries written = k_l - k_{l-1}; 0 if the worker hit a device error  */
+    int32_t*  level;   /* [M] sampled level l*, or -1 on a device error                            */
+    double*   p_sel;   /* [M] probability of the sampled level                                     */
+    int64_t   capacity;/* entries per worker; max_l (k_l - k_{l-1}) always suffices                */
+} mlmc_topk_msgs;
+
+/* Bit-plane message batch (Sec. 3.1: the residual of the fixed-point code is the level's bit
+ * field plus a sign bit per entry; with the unit schedule b_l = l+1 that is 2 bits per entry).
+ * Worker m owns planes[m * (1+w_max) * words ..], words = ceil(d/32).  Plane 0 holds the raw sign
+ * bits, plane j = 1..w_l holds bit (w_l - j) of the field (most significant first); bit t of word w
+ * is coordinate 32 w + t; bits past d are 0; planes past 1 + w_l are not written. */
+typedef struct {
+    uint32_t* planes;  /* [M][1 + w_max][ceil(d/32)]                                               */
+    float*    gmax;    /* [M] max_i |g_i|, the normaliser sent with the message                    */
+    int32_t*  level;   /* [M] sampled level, or -1 on a device error                               */
+    double*   p_sel;   /* [M]                                                                      */
+    int32_t   w_max;   /* magnitude planes allocated per worker; need >= max_l (b_l - b_{l-1})     */
+} mlmc_bit_msgs;
+
+/* Allocates the scratch workspace for problems up to (d_max, M_max, L_max) on `device`.
+ * Synchronous.  L_max <= MLMC_MAX_LEVELS.  Returns MLMC_ERR_NOMEM / MLMC_ERR_CUDA on failure. */
+int mlmc_create(mlmc_ctx** ctx, int device, int64_t d_max, int M_max, int L_max);
+int mlmc_destroy(mlmc_ctx* ctx);
+
+/* Synchronises `stream`, returns the sticky device status (first error since the last call) and clears it. */
+int mlmc_get_status(mlmc_ctx* ctx, void* stream);
+
+/* Number of kernels this ctx has launched so far (host counter; for launch accounting). */
+int64_t mlmc_launch_count(const mlmc_ctx* ctx);
+
+/* The uniforms of the level draw for workers 0..M-1 at (seed, step), computed on the device and
+ * copied to u_host[M].  Synchronous; for checking the counter generator against known answers. */
+int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream);
+
+/* Level probabilities and residual norms (Lemma 3.4; Alg. 3 "Compute p^l = Delta^l / sum Delta").
+ *   kind   MLMC_TOPK: sched = host int64 k[L];  MLMC_BITWISE: sched = host int64 b[L].
+ *   p_host NULL: adaptive, p_out[m][l] = Delta_l / sum Delta (all weight on level 0 if every Delta is 0).
+ *          else: host double[L], all > 0, sum 1 within 1e-9; p_out[m][l] = p_host[l] / sum.
+ *   p_out     device double [M][L].
+ *   delta_out device double [M][L] or NULL: Delta_l = ||C^l(g) - C^{l-1}(g)||_2 (always computed from g). */
+int mlmc_level_probs(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int kind,
+                     const int64_t* sched, int L, const double* p_host, double* p_out, double* delta_out,
+                     void* stream);
+
+/* MLMC-Top-k message of every worker (Alg. 2 / Alg. 3, the lines from "Sample l" to "Send").
+ *   k host int64[L], nondecreasing, k[L-1] = d (Def. 3.1: the top level is the identity).
+ *   p host double[L] or NULL for adaptive.  (seed, step, row index m) select the uniform of worker m.
+ * Device errors: capacity < band size -> MLMC_ERR_CAPACITY; NaN/Inf -> MLMC_ERR_NONFINITE. */
+int mlmc_compress_topk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld,
+                       const int64_t* k, int L, const double* p, uint64_t seed, uint64_t step,
+                       const mlmc_topk_msgs* out, void* stream);
+
+/* MLMC fixed-point bit-wise message of every worker (Sec. 3.1).
+ *   b host int32[L], strictly increasing, b[L-1] = B <= 23.
+ *   Code: e_i = fl32(|g_i| / gmax) (IEEE division), q_i = min(floor(e_i 2^B), 2^B - 1);
+ *   level l keeps the top b_l bits of q; field f_l = (q >> (B - b_l)) & (2^{w_l} - 1), w_l = b_l - b_{l-1};
+ *   residual entry = sign_i f_l 2^{-b_l} gmax;  adaptive Delta_l = gmax 2^{-b_l} sqrt(sum_i f_l^2). */
+int mlmc_compress_bitwise(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld,
+                          const int32_t* b, int L, const double* p, uint64_t seed, uint64_t step,
+                          const mlmc_bit_msgs* out, void* stream);
+
+/* Server average (Alg. 2 / Alg. 3 "Server aggregates: (1/M) sum_i g~_i") into dense out[d] (fp32,
+ * every element written exactly once).  kind selects the message struct msgs points to (host
+ * struct holding device pointers).  b host int32[L] for MLMC_BITWISE, ignored for MLMC_TOPK.
+ * Terms are added in worker order 0..M-1 in fp32, so the result is reproducible run to run.
+ * Workers whose level is -1 contribute nothing. */
+int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, int L, int M, int64_t d,
+                   float* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MLMC_H */

@@ -1,0 +1,351 @@
+// C ABI of the MLMC compression library: context, argument checks and the launch sequences.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+using namespace mlmc;
+
+struct mlmc_ctx {
+    Workspace ws;
+    void* slab;
+    size_t slab_bytes;
+};
+
+namespace {
+
+struct SlabPlanner {
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        const size_t at = off;
+        off += (bytes + 255) & ~size_t(255);
+        return at;
+    }
+};
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+int check_common(const mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int L) {
+    if (!ctx || !g) return MLMC_ERR_ARG;
+    if (dtype != MLMC_F32 && dtype != MLMC_BF16) return MLMC_ERR_ARG;
+    if (d < 1 || d > ctx->ws.d_max || d >= (int64_t(1) << 32)) return MLMC_ERR_ARG;
+    if (M < 1 || M > ctx->ws.M_max) return MLMC_ERR_ARG;
+    if (L < 1 || L > ctx->ws.L_max) return MLMC_ERR_ARG;
+    if (ld < d) return MLMC_ERR_ARG;
+    const int64_t esize = (dtype == MLMC_BF16) ? 2 : 4;
+    if (reinterpret_cast<uintptr_t>(g) % 16 != 0) return MLMC_ERR_ARG;
+    if (M > 1 && (ld * esize) % 16 != 0) return MLMC_ERR_ARG;
+    return MLMC_OK;
+}
+
+int check_topk_schedule(const int64_t* k, int L, int64_t d) {
+    if (!k) return MLMC_ERR_ARG;
+    int64_t prev = 0;
+    for (int l = 0; l < L; ++l) {
+        if (k[l] < prev || k[l] > d) return MLMC_ERR_SCHEDULE;
+        prev = k[l];
+    }
+    return k[L - 1] == d ? MLMC_OK : MLMC_ERR_SCHEDULE;  // Def. 3.1: the top level is the identity
+}
+
+template <typename I>
+int check_bit_schedule(const I* b, int L, int32_t* b32) {
+    if (!b) return MLMC_ERR_ARG;
+    int64_t prev = 0;
+    for (int l = 0; l < L; ++l) {
+        if (b[l] <= prev || b[l] > 23) return MLMC_ERR_SCHEDULE;
+        prev = b[l];
+        b32[l] = (int32_t)b[l];
+    }
+    return MLMC_OK;
+}
+
+// Lemma 3.2 asks for non-zero probabilities; they are renormalised in fp64.
+int normalise_probs(const double* p, int L, double* out) {
+    double s = 0.0;
+    for (int l = 0; l < L; ++l) {
+        if (!(p[l] > 0.0) || !std::isfinite(p[l])) return MLMC_ERR_PROB;
+        s += p[l];
+    }
+    if (std::fabs(s - 1.0) > 1e-9) return MLMC_ERR_PROB;
+    for (int l = 0; l < L; ++l) out[l] = p[l] / s;
+    return MLMC_OK;
+}
+
+int finish(cudaError_t e) { return e == cudaSuccess ? MLMC_OK : MLMC_ERR_CUDA; }
+
+// Thresholds of every live query (sweep 1 + the two masked digit passes for fp32).
+void run_selection(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
+    launch_hist1(ws, g, dtype, d, M, ld, s);
+    launch_resolve1(ws, dtype, M, L, s);
+    if (dtype == MLMC_F32 && L > 1) {
+        launch_masked_pass(ws, g, d, M, ld, 2, s);
+        launch_resolve23(ws, M, L, 2, s);
+        launch_masked_pass(ws, g, d, M, ld, 3, s);
+        launch_resolve23(ws, M, L, 3, s);
+    }
+}
+
+void run_band_norms(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
+    if (dtype == MLMC_BF16)
+        launch_norm_from_hist_bf16(ws, M, L, s);
+    else
+        launch_norm_sweep(ws, g, d, M, ld, L, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max) {
+    if (!out || d_max < 1 || d_max >= (int64_t(1) << 32) || M_max < 1 || L_max < 1 || L_max > kMaxLevels)
+        return MLMC_ERR_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MLMC_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MLMC_ERR_CUDA;
+    if (configure_select_kernels() != MLMC_OK) return MLMC_ERR_CUDA;
+
+    mlmc_ctx* ctx = new (std::nothrow) mlmc_ctx();
+    if (!ctx) return MLMC_ERR_NOMEM;
+    Workspace& ws = ctx->ws;
+    ws.device = device;
+    ws.d_max = d_max;
+    ws.M_max = M_max;
+    ws.L_max = L_max;
+    ws.sm_count = prop.multiProcessorCount;
+    ws.launches = 0;
+    ws.norm_ctas = ws.sm_count * 4;
+    ws.stat_ctas = ws.sm_count * 4;
+    const int64_t emit_tiles = (d_max + kEmitTile - 1) / kEmitTile;
+    const int64_t agg_tiles = (d_max + kAggTile - 1) / kAggTile;
+    ws.max_tiles = emit_tiles * M_max;
+
+    SlabPlanner pl;
+    const size_t o_status = pl.take(sizeof(int));
+    const size_t o_werr = pl.take(sizeof(int) * M_max);
+    const size_t o_hist1 = pl.take(sizeof(uint32_t) * kBins1 * M_max);
+    const size_t o_table1 = pl.take((size_t)kBins1 * M_max);
+    const size_t o_hist2 = pl.take(sizeof(uint32_t) * kMaxQueries * kBins23 * M_max);
+    const size_t o_map2 = pl.take((size_t)kMaxQueries * kBins23 * M_max);
+    const size_t o_hist3 = pl.take(sizeof(uint32_t) * kMaxQueries * kBins23 * M_max);
+    const size_t o_queries = pl.take(sizeof(Query) * kMaxQueries * M_max);
+    const size_t o_band = pl.take(sizeof(double) * kMaxLevels * ws.norm_ctas * M_max);
+    const size_t o_k = pl.take(sizeof(int64_t) * kMaxLevels);
+    const size_t o_pfix = pl.take(sizeof(double) * kMaxLevels);
+    const size_t o_pall = pl.take(sizeof(double) * kMaxLevels * M_max);
+    const size_t o_dall = pl.take(sizeof(double) * kMaxLevels * M_max);
+    const size_t o_u = pl.take(sizeof(double) * M_max);
+    const size_t o_emit = pl.take(sizeof(EmitParams) * M_max);
+    const size_t o_tagg = pl.take(sizeof(TileRec) * ws.max_tiles);
+    const size_t o_tinc = pl.take(sizeof(TileRec) * ws.max_tiles);
+    const size_t o_tcnt = pl.take(sizeof(unsigned));
+    const size_t o_aggoff = pl.take(sizeof(uint32_t) * (agg_tiles + 1) * M_max);
+    const size_t o_gmax = pl.take(sizeof(uint32_t) * M_max);
+    const size_t o_S = pl.take(sizeof(unsigned long long) * kMaxLevels * ws.stat_ctas * M_max);
+    const size_t o_blevel = pl.take(sizeof(int32_t) * M_max);
+
+    ctx->slab_bytes = pl.off;
+    if (cudaMalloc(&ctx->slab, ctx->slab_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return MLMC_ERR_NOMEM;
+    }
+    if (cudaMemset(ctx->slab, 0, ctx->slab_bytes) != cudaSuccess) {
+        cudaFree(ctx->slab);
+        delete ctx;
+        return MLMC_ERR_CUDA;
+    }
+    char* base = static_cast<char*>(ctx->slab);
+    ws.status = reinterpret_cast<int*>(base + o_status);
+    ws.worker_err = reinterpret_cast<int*>(base + o_werr);
+    ws.hist1 = reinterpret_cast<uint32_t*>(base + o_hist1);
+    ws.table1 = reinterpret_cast<uint8_t*>(base + o_table1);
+    ws.hist2 = reinterpret_cast<uint32_t*>(base + o_hist2);
+    ws.map2 = reinterpret_cast<uint8_t*>(base + o_map2);
+    ws.hist3 = reinterpret_cast<uint32_t*>(base + o_hist3);
+    ws.queries = reinterpret_cast<Query*>(base + o_queries);
+    ws.band_partial = reinterpret_cast<double*>(base + o_band);
+    ws.k_dev = reinterpret_cast<int64_t*>(base + o_k);
+    ws.p_fixed = reinterpret_cast<double*>(base + o_pfix);
+    ws.p_all = reinterpret_cast<double*>(base + o_pall);
+    ws.delta_all = reinterpret_cast<double*>(base + o_dall);
+    ws.u_dev = reinterpret_cast<double*>(base + o_u);
+    ws.emit = reinterpret_cast<EmitParams*>(base + o_emit);
+    ws.tile_agg = reinterpret_cast<TileRec*>(base + o_tagg);
+    ws.tile_inc = reinterpret_cast<TileRec*>(base + o_tinc);
+    ws.tile_counter = reinterpret_cast<unsigned*>(base + o_tcnt);
+    ws.agg_offsets = reinterpret_cast<uint32_t*>(base + o_aggoff);
+    ws.gmax_bits = reinterpret_cast<uint32_t*>(base + o_gmax);
+    ws.S_partial = reinterpret_cast<unsigned long long*>(base + o_S);
+    ws.bit_level = reinterpret_cast<int32_t*>(base + o_blevel);
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        cudaFree(ctx->slab);
+        delete ctx;
+        return MLMC_ERR_CUDA;
+    }
+    *out = ctx;
+    return MLMC_OK;
+}
+
+int mlmc_destroy(mlmc_ctx* ctx) {
+    if (!ctx) return MLMC_ERR_ARG;
+    DeviceGuard guard(ctx->ws.device);
+    cudaDeviceSynchronize();
+    const cudaError_t e = cudaFree(ctx->slab);
+    delete ctx;
+    return finish(e);
+}
+
+int mlmc_get_status(mlmc_ctx* ctx, void* stream) {
+    if (!ctx) return MLMC_ERR_ARG;
+    DeviceGuard guard(ctx->ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int st = 0;
+    if (cudaMemcpyAsync(&st, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return MLMC_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MLMC_ERR_CUDA;
+    if (st != 0) {
+        if (cudaMemsetAsync(ctx->ws.status, 0, sizeof(int), s) != cudaSuccess) return MLMC_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return MLMC_ERR_CUDA;
+    }
+    return st;
+}
+
+int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches : 0; }
+
+int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream) {
+    if (!ctx || !u_host || M < 1 || M > ctx->ws.M_max) return MLMC_ERR_ARG;
+    DeviceGuard guard(ctx->ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    launch_uniforms(ctx->ws, M, seed, step, s);
+    if (cudaMemcpyAsync(u_host, ctx->ws.u_dev, sizeof(double) * M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    return finish(cudaStreamSynchronize(s));
+}
+
+int mlmc_level_probs(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int kind,
+                     const int64_t* sched, int L, const double* p_host, double* p_out, double* delta_out,
+                     void* stream) {
+    if (int rc = check_common(ctx, g, dtype, d, M, ld, L)) return rc;
+    if (!p_out || (kind != MLMC_TOPK && kind != MLMC_BITWISE)) return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    double pn[kMaxLevels];
+    int32_t b32[kMaxLevels];
+    if (kind == MLMC_TOPK) {
+        if (int rc = check_topk_schedule(sched, L, d)) return rc;
+    } else {
+        if (int rc = check_bit_schedule(sched, L, b32)) return rc;
+    }
+    if (p_host)
+        if (int rc = normalise_probs(p_host, L, pn)) return rc;
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+    if (p_host) cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
+    const bool need_data = (p_host == nullptr) || (delta_out != nullptr);
+    if (kind == MLMC_TOPK) {
+        cudaMemcpyAsync(ws.k_dev, sched, sizeof(int64_t) * L, cudaMemcpyHostToDevice, s);
+        if (need_data) {
+            launch_init_queries_adaptive(ws, M, L, d, s);
+            run_selection(ws, g, dtype, d, M, ld, L, s);
+            run_band_norms(ws, g, dtype, d, M, ld, L, s);
+            launch_probs_draw(ws, dtype, M, L, d, true, false, 0, 0, nullptr, s);
+        }
+    } else {
+        if (need_data) {
+            launch_absmax(ws, g, dtype, d, M, ld, s);
+            launch_bit_stats(ws, g, dtype, d, M, ld, b32, L, s);
+            launch_bit_probs_draw(ws, M, b32, L, true, true, 0, 0, nullptr, s);
+        }
+    }
+    launch_copy_probs(ws, M, L, p_host ? ws.p_fixed : nullptr, p_out, delta_out, s);
+    return finish(cudaGetLastError());
+}
+
+int mlmc_compress_topk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, const int64_t* k,
+                       int L, const double* p, uint64_t seed, uint64_t step, const mlmc_topk_msgs* out,
+                       void* stream) {
+    if (int rc = check_common(ctx, g, dtype, d, M, ld, L)) return rc;
+    if (!out || !out->idx || !out->val || !out->count || !out->level || !out->p_sel || out->capacity < 0)
+        return MLMC_ERR_ARG;
+    if (int rc = check_topk_schedule(k, L, d)) return rc;
+    double pn[kMaxLevels];
+    if (p)
+        if (int rc = normalise_probs(p, L, pn)) return rc;
+    Workspace& ws = ctx->ws;
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+    cudaMemcpyAsync(ws.k_dev, k, sizeof(int64_t) * L, cudaMemcpyHostToDevice, s);
+    const bool adaptive = (p == nullptr);
+    if (adaptive) {
+        launch_init_queries_adaptive(ws, M, L, d, s);
+    } else {
+        cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
+        launch_draw_fixed(ws, M, L, d, seed, step, s);  // the draw does not depend on the data: only two thresholds are needed
+    }
+    run_selection(ws, g, dtype, d, M, ld, L, s);
+    if (adaptive) run_band_norms(ws, g, dtype, d, M, ld, L, s);
+    launch_probs_draw(ws, dtype, M, L, d, adaptive, true, seed, step, out, s);
+    launch_emit(ws, g, dtype, d, M, ld, *out, s);
+    return finish(cudaGetLastError());
+}
+
+int mlmc_compress_bitwise(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b,
+                          int L, const double* p, uint64_t seed, uint64_t step, const mlmc_bit_msgs* out,
+                          void* stream) {
+    if (int rc = check_common(ctx, g, dtype, d, M, ld, L)) return rc;
+    if (!out || !out->planes || !out->gmax || !out->level || !out->p_sel || out->w_max < 1) return MLMC_ERR_ARG;
+    int32_t b32[kMaxLevels];
+    if (int rc = check_bit_schedule(b, L, b32)) return rc;
+    double pn[kMaxLevels];
+    if (p)
+        if (int rc = normalise_probs(p, L, pn)) return rc;
+    Workspace& ws = ctx->ws;
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+    const bool adaptive = (p == nullptr);
+    if (!adaptive) cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
+    launch_absmax(ws, g, dtype, d, M, ld, s);
+    if (adaptive) launch_bit_stats(ws, g, dtype, d, M, ld, b32, L, s);
+    launch_bit_probs_draw(ws, M, b32, L, adaptive, false, seed, step, out, s);
+    launch_bit_pack(ws, g, dtype, d, M, ld, b32, L, *out, s);
+    return finish(cudaGetLastError());
+}
+
+int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, int L, int M, int64_t d, float* out,
+                   void* stream) {
+    if (!ctx || !msgs || !out) return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    if (d < 1 || d > ws.d_max || M < 1 || M > ws.M_max) return MLMC_ERR_ARG;
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (kind == MLMC_TOPK) {
+        const mlmc_topk_msgs* t = static_cast<const mlmc_topk_msgs*>(msgs);
+        if (!t->idx || !t->val || !t->count || !t->level) return MLMC_ERR_ARG;
+        launch_aggregate_topk(ws, *t, M, d, out, s);
+    } else if (kind == MLMC_BITWISE) {
+        const mlmc_bit_msgs* t = static_cast<const mlmc_bit_msgs*>(msgs);
+        if (!t->planes || !t->gmax || !t->level || !t->p_sel || L < 1 || L > kMaxLevels) return MLMC_ERR_ARG;
+        int32_t b32[kMaxLevels];
+        if (int rc = check_bit_schedule(b, L, b32)) return rc;
+        launch_aggregate_bitwise(ws, *t, b32, L, M, d, out, s);
+    } else {
+        return MLMC_ERR_ARG;
+    }
+    return finish(cudaGetLastError());
+}
+
+}  // extern "C"

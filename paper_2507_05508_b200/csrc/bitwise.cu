@@ -1,0 +1,393 @@
+// MLMC with the fixed-point bit-wise compressor (Sec. 3.1).
+//
+// Entries are divided by the largest magnitude of the worker's gradient and written as a sign plus
+// B fractional bits (Eq. 6 with B = b_{L-1} <= 23 instead of 63, since the input is fp32/bf16):
+//   e = fl32(|g| / gmax),  q = min(floor(e 2^B), 2^B - 1).
+// Level l keeps the top b_l bits of q; the residual C^l - C^{l-1} is the field
+//   f_l = (q >> (B - b_l)) & (2^{w_l} - 1),  w_l = b_l - b_{l-1},  worth  sign f_l 2^{-b_l} gmax,
+// sent as one sign plane and w_l magnitude planes.  Adaptive probabilities (Lemma 3.4) use the exact
+// integer field energies S_l = sum_i f_l^2:  Delta_l = gmax 2^{-b_l} sqrt(S_l).
+#include "common.cuh"
+
+namespace mlmc {
+
+namespace {
+
+constexpr int kBitThreads = 256;
+
+struct BitSchedule {
+    int L;
+    int B;
+    int shift[kMaxLevels];      // B - b_l
+    uint32_t mask[kMaxLevels];  // 2^{w_l} - 1
+    int width[kMaxLevels];      // w_l
+    int bits[kMaxLevels];       // b_l
+};
+
+__device__ __forceinline__ uint32_t fixed_point_code(float mag, float gmax, float two_b, uint32_t qmax) {
+    const float e = __fdiv_rn(mag, gmax);        // IEEE division: "divide the entries by the largest entry"
+    const float scaled = __fmul_rn(e, two_b);    // exact power-of-two scaling
+    const uint32_t q = __float2uint_rz(scaled);  // truncation: the lower bits are discarded
+    return min(q, qmax);
+}
+
+// ---- per-worker max |g| as an integer max over magnitude keys; flags NaN / Inf
+template <typename T>
+__global__ void __launch_bounds__(kSweepThreads)
+absmax_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* gmax_bits, int* status, int* worker_err) {
+    using Tr = ElemTraits<T>;
+    __shared__ uint32_t sh_max[kSweepThreads / 32];
+    const int m = blockIdx.y;
+    const T* row = g + (int64_t)m * ld;
+    int64_t v0, v1;
+    block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
+    uint32_t mx = 0;
+#pragma unroll 4
+    for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x)
+        for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) { mx = max(mx, Tr::key(bits)); });
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    if ((threadIdx.x & 31) == 0) sh_max[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kSweepThreads / 32; ++w) mx = max(mx, sh_max[w]);
+        if (mx >= Tr::kInfKey) {
+            worker_err[m] = MLMC_ERR_NONFINITE;
+            set_status(status, MLMC_ERR_NONFINITE);
+        }
+        const uint32_t as_f32 = (Tr::kVec == 8) ? (mx << 16) : mx;
+        atomicMax(&gmax_bits[m], as_f32);
+    }
+}
+
+// ---- adaptive only: exact field energies S_l = sum_i f_l^2 for every level in one sweep
+template <typename T, int LMAX>
+__global__ void __launch_bounds__(kSweepThreads)
+bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* __restrict__ gmax_bits,
+                 BitSchedule sc, unsigned long long* __restrict__ S_partial, int stat_ctas, const int* worker_err) {
+    using Tr = ElemTraits<T>;
+    __shared__ unsigned long long sh_red[kSweepThreads / 32];
+    const int m = blockIdx.y;
+    if (worker_err[m]) return;
+    const float gmax = __uint_as_float(gmax_bits[m]);
+    const float two_b = (float)(1u << sc.B);
+    const uint32_t qmax = (1u << sc.B) - 1u;
+    unsigned long long acc[LMAX];
+#pragma unroll
+    for (int l = 0; l < LMAX; ++l) acc[l] = 0;
+    if (gmax > 0.0f) {
+        const T* row = g + (int64_t)m * ld;
+        int64_t v0, v1;
+        block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
+#pragma unroll 2
+        for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+            for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) {
+                const float mag = fabsf(Tr::value(bits));
+                const uint32_t q = fixed_point_code(mag, gmax, two_b, qmax);
+#pragma unroll
+                for (int l = 0; l < LMAX; ++l) {
+                    if (l < sc.L) {
+                        const uint32_t f = (q >> sc.shift[l]) & sc.mask[l];
+                        acc[l] += (unsigned long long)f * f;
+                    }
+                }
+            });
+        }
+    }
+#pragma unroll
+    for (int l = 0; l < LMAX; ++l) {
+        if (l >= sc.L) break;
+        unsigned long long x = acc[l];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        if ((threadIdx.x & 31) == 0) sh_red[threadIdx.x >> 5] = x;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long s = 0;
+            for (int w = 0; w < kSweepThreads / 32; ++w) s += sh_red[w];
+            S_partial[((int64_t)m * stat_ctas + blockIdx.x) * kMaxLevels + l] = s;
+        }
+        __syncthreads();
+    }
+}
+
+__device__ int draw_level_bits(const double* p, int L, double u) {
+    int j_last = -1;
+    for (int j = 0; j < L; ++j)
+        if (p[j] > 0.0) j_last = j;
+    double c = 0.0;
+    for (int j = 0; j < L; ++j) {
+        c += p[j];
+        const double cdf = (j >= j_last) ? 1.0 : c;
+        if (u < cdf) return j;
+    }
+    return 0;
+}
+
+// ---- probabilities, draw and message header of every worker (one thread per worker)
+__global__ void bit_probs_draw_kernel(BitSchedule sc, const uint32_t* gmax_bits, const unsigned long long* S_partial,
+                                      int n_partials, int stat_ctas, const double* p_fixed, int adaptive,
+                                      int need_delta, uint64_t seed, uint64_t step, int M, double* p_all,
+                                      double* delta_all, double* u_dev, int32_t* bit_level, float* out_gmax,
+                                      int32_t* out_level, double* out_p_sel, int w_max, int want_msg, int* status,
+                                      int* worker_err) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= M) return;
+    if (worker_err[m]) {
+        bit_level[m] = -1;
+        if (want_msg) {
+            out_level[m] = -1;
+            out_p_sel[m] = 0.0;
+            out_gmax[m] = 0.0f;
+        }
+        return;
+    }
+    const float gmax = __uint_as_float(gmax_bits[m]);
+    double p[kMaxLevels], delta[kMaxLevels];
+    if (adaptive || need_delta) {
+        for (int l = 0; l < sc.L; ++l) {
+            // exact 128-bit sum of the per-block partials, rounded once to fp64
+            unsigned __int128 S = 0;
+            for (int c = 0; c < n_partials; ++c) S += S_partial[((int64_t)m * stat_ctas + c) * kMaxLevels + l];
+            const double Sd = (double)(unsigned long long)(S >> 64) * 0x1.0p64 + (double)(unsigned long long)S;
+            delta[l] = (double)gmax * ldexp(1.0, -sc.bits[l]) * sqrt(Sd);
+            delta_all[m * kMaxLevels + l] = delta[l];
+        }
+    }
+    if (adaptive) {
+        double s = 0.0;
+        for (int l = 0; l < sc.L; ++l) s += delta[l];
+        for (int l = 0; l < sc.L; ++l) p[l] = (s > 0.0) ? delta[l] / s : (l == 0 ? 1.0 : 0.0);
+    } else {
+        for (int l = 0; l < sc.L; ++l) p[l] = p_fixed[l];
+    }
+    for (int l = 0; l < sc.L; ++l) p_all[m * kMaxLevels + l] = p[l];
+    const double u = counter_uniform(seed, step, (uint64_t)m);
+    u_dev[m] = u;
+    int level = draw_level_bits(p, sc.L, u);
+    if (want_msg) {
+        if (sc.width[level] > w_max) {
+            worker_err[m] = MLMC_ERR_CAPACITY;
+            set_status(status, MLMC_ERR_CAPACITY);
+            level = -1;
+        }
+        out_level[m] = level;
+        out_p_sel[m] = (level >= 0) ? p[level] : 0.0;
+        out_gmax[m] = gmax;
+    }
+    bit_level[m] = level;
+}
+
+// ---- pack: every warp turns 1024 consecutive entries into 32 words of each plane
+template <typename T>
+__global__ void __launch_bounds__(kBitThreads)
+bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* __restrict__ gmax_bits,
+                BitSchedule sc, const int32_t* __restrict__ bit_level, uint32_t* __restrict__ planes, int w_max,
+                int64_t words) {
+    using Tr = ElemTraits<T>;
+    const int m = blockIdx.y;
+    const int level = bit_level[m];
+    if (level < 0) return;
+    const int lane = threadIdx.x & 31;
+    const int warps_per_block = kBitThreads / 32;
+    const int64_t ngroups = (words + 31) / 32;  // groups of 32 words = 1024 entries
+    const float gmax = __uint_as_float(gmax_bits[m]);
+    const float two_b = (float)(1u << sc.B);
+    const uint32_t qmax = (1u << sc.B) - 1u;
+    const int shift = sc.shift[level];
+    const uint32_t mask = sc.mask[level];
+    const int w = sc.width[level];
+    const T* row = g + (int64_t)m * ld;
+    uint32_t* out = planes + (int64_t)m * (1 + w_max) * words;
+    for (int64_t grp = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); grp < ngroups;
+         grp += (int64_t)gridDim.x * warps_per_block) {
+        const int64_t e0 = grp * 1024;
+        uint32_t code[32];  // bit 31 = sign, low bits = field
+#pragma unroll
+        for (int s = 0; s < 32; ++s) {
+            const int64_t i = e0 + s * 32 + lane;
+            uint32_t c = 0;
+            if (i < d) {
+                uint32_t bits;
+                if constexpr (Tr::kVec == 4)
+                    bits = __ldg(reinterpret_cast<const uint32_t*>(row) + i);
+                else
+                    bits = __ldg(reinterpret_cast<const uint16_t*>(row) + i);
+                const float x = Tr::value(bits);
+                const uint32_t q = (gmax > 0.0f) ? fixed_point_code(fabsf(x), gmax, two_b, qmax) : 0u;
+                c = ((q >> shift) & mask) | (__float_as_uint(x) & 0x80000000u);
+            }
+            code[s] = c;
+        }
+        const int64_t word = grp * 32 + lane;
+        for (int j = 0; j <= w; ++j) {
+            const int bit = (j == 0) ? 31 : (w - j);
+            uint32_t mine = 0;
+#pragma unroll
+            for (int s = 0; s < 32; ++s) {
+                const uint32_t b = __ballot_sync(0xFFFFFFFFu, (code[s] >> bit) & 1u);
+                if (lane == s) mine = b;
+            }
+            if (word < words) out[(int64_t)j * words + word] = mine;
+        }
+    }
+}
+
+// ---- server average of bit-plane messages: thread = one word (32 entries), staged through shared memory
+__global__ void __launch_bounds__(kBitThreads)
+aggregate_bitwise_kernel(const uint32_t* __restrict__ planes, const float* __restrict__ gmax,
+                         const int32_t* __restrict__ level, const double* __restrict__ p_sel, BitSchedule sc,
+                         int w_max, int64_t words, int M, int64_t d, float* __restrict__ out) {
+    __shared__ float sh_out[kBitThreads / 32][32][33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float fM = (float)M;
+    const int64_t nblk = (words + kBitThreads - 1) / kBitThreads;
+    for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
+        const int64_t word = blk * kBitThreads + threadIdx.x;
+        float acc[32];
+#pragma unroll
+        for (int t = 0; t < 32; ++t) acc[t] = 0.0f;
+        for (int m = 0; m < M; ++m) {  // fixed worker order
+            const int lv = level[m];
+            if (lv < 0) continue;
+            const int w = sc.width[lv];
+            // value of one unit of the field: 2^{-b_l} gmax / p_l
+            const float unit = (float)(ldexp((double)gmax[m], -sc.bits[lv]) / p_sel[m]);
+            const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
+            const uint32_t sgn = (word < words) ? pm[word] : 0u;
+            uint32_t f[32];
+#pragma unroll
+            for (int t = 0; t < 32; ++t) f[t] = 0;
+            for (int j = 1; j <= w; ++j) {
+                const uint32_t pw = (word < words) ? pm[(int64_t)j * words + word] : 0u;
+#pragma unroll
+                for (int t = 0; t < 32; ++t) f[t] = (f[t] << 1) | ((pw >> t) & 1u);
+            }
+#pragma unroll
+            for (int t = 0; t < 32; ++t) {
+                const float v = (float)f[t] * unit;
+                acc[t] += ((sgn >> t) & 1u) ? -v : v;
+            }
+        }
+        // transpose through shared memory so that the 32 floats of a word leave as one 128-byte row
+#pragma unroll
+        for (int t = 0; t < 32; ++t) sh_out[warp][lane][t] = acc[t] / fM;
+        __syncwarp();
+        const int64_t wbase = blk * kBitThreads + warp * 32;
+#pragma unroll 4
+        for (int r = 0; r < 32; ++r) {
+            const int64_t i = (wbase + r) * 32 + lane;
+            if (i < d) out[i] = sh_out[warp][r][lane];
+        }
+        __syncwarp();
+    }
+}
+
+BitSchedule make_schedule(const int32_t* b, int L) {
+    BitSchedule sc = {};
+    sc.L = L;
+    sc.B = b[L - 1];
+    for (int l = 0; l < L; ++l) {
+        const int w = b[l] - (l ? b[l - 1] : 0);
+        sc.bits[l] = b[l];
+        sc.width[l] = w;
+        sc.shift[l] = sc.B - b[l];
+        sc.mask[l] = (w >= 32) ? 0xFFFFFFFFu : ((1u << w) - 1u);
+    }
+    return sc;
+}
+
+int bit_blocks(const Workspace& ws, int64_t d, int vec, int M, int waves) {
+    const int64_t nvec = (d + vec - 1) / vec;
+    const int64_t by_work = (nvec + (int64_t)kSweepThreads * 4 - 1) / ((int64_t)kSweepThreads * 4);
+    int64_t by_sm = ((int64_t)ws.sm_count * waves + M - 1) / M;
+    int64_t nb = by_work < by_sm ? by_work : by_sm;
+    return (int)(nb < 1 ? 1 : nb);
+}
+
+}  // namespace
+
+void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
+    cudaMemsetAsync(ws.gmax_bits, 0, (size_t)M * sizeof(uint32_t), s);
+    if (dtype == MLMC_BF16) {
+        const int nb = bit_blocks(ws, d, 8, M, 8);
+        absmax_kernel<bf16_t><<<dim3(nb, M), kSweepThreads, 0, s>>>(static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits,
+                                                                    ws.status, ws.worker_err);
+    } else {
+        const int nb = bit_blocks(ws, d, 4, M, 8);
+        absmax_kernel<float><<<dim3(nb, M), kSweepThreads, 0, s>>>(static_cast<const float*>(g), d, ld, ws.gmax_bits,
+                                                                   ws.status, ws.worker_err);
+    }
+    ws.launches++;
+}
+
+template <typename T>
+static void launch_bit_stats_t(Workspace& ws, const T* g, int64_t d, int M, int64_t ld, const BitSchedule& sc, int nb,
+                               cudaStream_t s) {
+    dim3 grid(nb, M);
+    if (sc.L <= 8)
+        bit_stats_kernel<T, 8><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas,
+                                                              ws.worker_err);
+    else if (sc.L <= 16)
+        bit_stats_kernel<T, 16><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas,
+                                                               ws.worker_err);
+    else
+        bit_stats_kernel<T, 23><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas,
+                                                               ws.worker_err);
+}
+
+void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
+                      cudaStream_t s) {
+    const BitSchedule sc = make_schedule(b, L);
+    cudaMemsetAsync(ws.S_partial, 0, (size_t)M * ws.stat_ctas * kMaxLevels * sizeof(unsigned long long), s);
+    int nb = bit_blocks(ws, d, dtype == MLMC_BF16 ? 8 : 4, M, 4);
+    if (nb > ws.stat_ctas) nb = ws.stat_ctas;
+    if (dtype == MLMC_BF16)
+        launch_bit_stats_t<bf16_t>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, nb, s);
+    else
+        launch_bit_stats_t<float>(ws, static_cast<const float*>(g), d, M, ld, sc, nb, s);
+    ws.launches++;
+}
+
+void launch_bit_probs_draw(Workspace& ws, int M, const int32_t* b, int L, bool adaptive, bool need_delta,
+                           uint64_t seed, uint64_t step, const mlmc_bit_msgs* out, cudaStream_t s) {
+    const BitSchedule sc = make_schedule(b, L);
+    bit_probs_draw_kernel<<<(M + 63) / 64, 64, 0, s>>>(
+        sc, ws.gmax_bits, ws.S_partial, ws.stat_ctas, ws.stat_ctas, ws.p_fixed, adaptive ? 1 : 0, need_delta ? 1 : 0,
+        seed, step, M, ws.p_all, ws.delta_all, ws.u_dev, ws.bit_level, out ? out->gmax : nullptr,
+        out ? out->level : nullptr, out ? out->p_sel : nullptr, out ? out->w_max : 0, out ? 1 : 0, ws.status,
+        ws.worker_err);
+    ws.launches++;
+}
+
+void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
+                     const mlmc_bit_msgs& out, cudaStream_t s) {
+    const BitSchedule sc = make_schedule(b, L);
+    const int64_t words = (d + 31) / 32;
+    const int64_t ngroups = (words + 31) / 32;
+    int64_t nb = (ngroups + (kBitThreads / 32) - 1) / (kBitThreads / 32);
+    const int64_t cap = ((int64_t)ws.sm_count * 16 + M - 1) / M;
+    if (nb > cap) nb = cap;
+    if (nb < 1) nb = 1;
+    if (dtype == MLMC_BF16)
+        bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, 0, s>>>(
+            static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
+    else
+        bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, 0, s>>>(
+            static_cast<const float*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
+    ws.launches++;
+}
+
+void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const int32_t* b, int L, int M, int64_t d,
+                              float* out, cudaStream_t s) {
+    const BitSchedule sc = make_schedule(b, L);
+    const int64_t words = (d + 31) / 32;
+    int64_t nb = (words + kBitThreads - 1) / kBitThreads;
+    const int64_t cap = (int64_t)ws.sm_count * 8;
+    if (nb > cap) nb = cap;
+    aggregate_bitwise_kernel<<<(unsigned)nb, kBitThreads, 0, s>>>(msgs.planes, msgs.gmax, msgs.level, msgs.p_sel, sc,
+                                                                  msgs.w_max, words, M, d, out);
+    ws.launches++;
+}
+
+}  // namespace mlmc

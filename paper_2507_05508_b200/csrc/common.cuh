@@ -1,0 +1,212 @@
+// Shared declarations of the MLMC CUDA library: workspace layout, device helpers, launcher prototypes.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mlmc.h"
+
+namespace mlmc {
+
+constexpr int kMaxLevels = MLMC_MAX_LEVELS;   // L <= 32, so at most 31 thresholds per worker
+constexpr int kMaxQueries = kMaxLevels;
+constexpr int kBins1 = 32768;                 // leading digit: key bits 30..16 (fp32) / the whole key (bf16)
+constexpr int kBins23 = 256;                  // second and third digits: key bits 15..8 and 7..0
+constexpr uint32_t kKeyNone = 0xFFFFFFFFu;    // threshold above every finite key: "nothing is inside"
+constexpr uint32_t kNoSlot = 0xFFu;
+
+constexpr int kSweepThreads = 512;            // histogram / masked / norm sweeps
+constexpr int kEmitThreads = 256;
+constexpr int kEmitItems = 16;                // elements per thread per tile
+constexpr int kEmitTile = kEmitThreads * kEmitItems;
+constexpr int kAggTile = 4096;                // dense output elements per aggregation tile
+
+// Per-worker selection query: the rank-k element of the total order.
+struct Query {
+    uint32_t k;        // target rank, 1 <= k < d for live queries
+    uint32_t prefix;   // key bits fixed so far
+    uint32_t rem;      // rank still to descend inside the current prefix set (1-based, from the top)
+    uint32_t slot;     // histogram slot of the next digit pass (kNoSlot when resolved or trivial)
+    uint32_t T;        // resolved threshold key
+    uint32_t c;        // #{ key > T }
+    uint32_t n;        // #{ key == T }
+    uint32_t r;        // how many key == T elements, in index order, are inside Top-k  (k - c)
+    uint32_t trivial;  // 1: k == 0 (nothing inside), 2: k >= d (everything inside), 0: live
+    uint32_t pad[3];
+};
+
+// Emit parameters of one worker, produced by the draw kernel.
+struct EmitParams {
+    uint32_t Ta, ra;   // Top-k_{l*-1}: inside iff key > Ta or (key == Ta and tie rank <= ra)
+    uint32_t Tb, rb;   // Top-k_{l*}
+    double inv_p;      // 1 / p_{l*}
+    uint32_t expect;   // k_{l*} - k_{l*-1}
+    int32_t enabled;   // 0: worker skipped (device error)
+    int32_t level;
+    int32_t pad;
+};
+
+// Look-back record of one emit tile: three running counts published once each.
+struct TileRec {
+    uint32_t D, Ea, Eb;
+    uint32_t flag;
+};
+
+struct Workspace {
+    int device;
+    int64_t d_max;
+    int M_max, L_max;
+    int sm_count;
+    int64_t launches;
+    // device memory
+    int* status;                 // sticky status word
+    int* worker_err;             // [M] per-worker device error (0 = fine)
+    uint32_t* hist1;             // [M][kBins1]  counts, then suffix sums in place
+    uint8_t* table1;             // [M][kBins1]  leading-digit bin -> slot of pass 2
+    uint32_t* hist2;             // [M][kMaxQueries][256]
+    uint8_t* map2;               // [M][kMaxQueries][256] (slot2, digit2) -> slot of pass 3
+    uint32_t* hist3;             // [M][kMaxQueries][256]
+    Query* queries;              // [M][kMaxQueries]
+    double* band_partial;        // [M][norm_ctas][kMaxLevels] per-block open-interval sums
+    int norm_ctas;
+    int64_t* k_dev;              // [kMaxLevels] schedule
+    double* p_fixed;             // [kMaxLevels] normalised fixed p
+    double* p_all;               // [M][kMaxLevels]
+    double* delta_all;           // [M][kMaxLevels]
+    double* u_dev;               // [M]
+    EmitParams* emit;            // [M]
+    TileRec* tile_agg;           // [max_tiles]
+    TileRec* tile_inc;           // [max_tiles]
+    int64_t max_tiles;
+    unsigned int* tile_counter;  // dynamic tile ticket
+    uint32_t* agg_offsets;       // [M][agg_tiles_max + 1]
+    // bit-wise
+    uint32_t* gmax_bits;         // [M]
+    unsigned long long* S_partial;  // [M][stat_ctas][kMaxLevels]
+    int stat_ctas;
+    int32_t* bit_level;          // [M] (mirrors out->level for the pack kernel)
+};
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+__device__ __forceinline__ uint64_t splitmix_finalize(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// One uniform in [0,1) per (seed, step, worker): three chained SplitMix64 output rounds.
+__device__ __forceinline__ double counter_uniform(uint64_t seed, uint64_t step, uint64_t worker) {
+    const uint64_t golden = 0x9E3779B97F4A7C15ull;
+    uint64_t h = splitmix_finalize(seed + golden);
+    h = splitmix_finalize(h + step + golden);
+    h = splitmix_finalize(h + worker + golden);
+    return (double)(h >> 11) * 0x1.0p-53;
+}
+
+// Magnitude key: monotone in |g| for finite values.  fp32: 31 bits; bf16: 15 bits.
+template <typename T>
+struct ElemTraits;
+
+template <>
+struct ElemTraits<float> {
+    static constexpr int kVec = 4;             // elements per 16-byte load
+    static constexpr uint32_t kInfKey = 0x7F800000u;
+    static constexpr int kShift1 = 16;         // key >> kShift1 = leading digit
+    __device__ static __forceinline__ uint32_t key(uint32_t bits) { return bits & 0x7FFFFFFFu; }
+    __device__ static __forceinline__ float value(uint32_t bits) { return __uint_as_float(bits); }
+};
+
+struct bf16_t {
+    uint16_t x;
+};
+
+template <>
+struct ElemTraits<bf16_t> {
+    static constexpr int kVec = 8;
+    static constexpr uint32_t kInfKey = 0x7F80u;
+    static constexpr int kShift1 = 0;
+    __device__ static __forceinline__ uint32_t key(uint32_t bits) { return bits & 0x7FFFu; }
+    __device__ static __forceinline__ float value(uint32_t bits) { return __uint_as_float(bits << 16); }
+};
+
+// Loads the 16-byte vector v of a row and hands each element's raw bits to f(index_in_row, bits).
+// Elements at or past d are skipped; a vector that straddles d is read element by element.
+template <typename T, typename F>
+__device__ __forceinline__ void for_each_in_vector(const T* row, int64_t v, int64_t d, F&& f) {
+    constexpr int V = ElemTraits<T>::kVec;
+    const int64_t base = v * V;
+    if (base + V <= d) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + v);
+        if constexpr (V == 4) {
+            f(base + 0, q.x);
+            f(base + 1, q.y);
+            f(base + 2, q.z);
+            f(base + 3, q.w);
+        } else {
+            f(base + 0, q.x & 0xFFFFu);
+            f(base + 1, q.x >> 16);
+            f(base + 2, q.y & 0xFFFFu);
+            f(base + 3, q.y >> 16);
+            f(base + 4, q.z & 0xFFFFu);
+            f(base + 5, q.z >> 16);
+            f(base + 6, q.w & 0xFFFFu);
+            f(base + 7, q.w >> 16);
+        }
+    } else {
+        for (int64_t i = base; i < d; ++i) {
+            uint32_t bits;
+            if constexpr (V == 4)
+                bits = reinterpret_cast<const uint32_t*>(row)[i];
+            else
+                bits = reinterpret_cast<const uint16_t*>(row)[i];
+            f(i, bits);
+        }
+    }
+}
+
+// Contiguous range of 16-byte vectors handled by block `bx` of `nb` blocks over a row of d elements.
+__device__ __forceinline__ void block_vector_range(int64_t d, int vec, int bx, int nb, int64_t* v0, int64_t* v1) {
+    const int64_t nvec = (d + vec - 1) / vec;
+    const int64_t per = (nvec + nb - 1) / nb;
+    *v0 = min((int64_t)bx * per, nvec);
+    *v1 = min(*v0 + per, nvec);
+}
+
+// ---------------------------------------------------------------------------------------------
+// launchers (each enqueues on `s` and bumps ws.launches)
+// ---------------------------------------------------------------------------------------------
+// topk_select.cu
+int configure_select_kernels();
+void launch_init_queries_adaptive(Workspace& ws, int M, int L, int64_t d, cudaStream_t s);
+void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, cudaStream_t s);
+void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStream_t s);
+void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s);
+void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s);
+void launch_masked_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s);
+void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s);
+void launch_norm_sweep(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s);
+void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s);
+void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool adaptive, bool want_emit,
+                       uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, cudaStream_t s);
+void launch_copy_probs(Workspace& ws, int M, int L, const double* p_fixed, double* p_out, double* delta_out,
+                       cudaStream_t s);
+// topk_emit.cu
+void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const mlmc_topk_msgs& out,
+                 cudaStream_t s);
+void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int64_t d, float* out, cudaStream_t s);
+// bitwise.cu
+void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s);
+void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
+                      cudaStream_t s);
+void launch_bit_probs_draw(Workspace& ws, int M, const int32_t* b, int L, bool adaptive, bool need_delta,
+                           uint64_t seed, uint64_t step, const mlmc_bit_msgs* out, cudaStream_t s);
+void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
+                     const mlmc_bit_msgs& out, cudaStream_t s);
+void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const int32_t* b, int L, int M, int64_t d,
+                              float* out, cudaStream_t s);
+
+}  // namespace mlmc

@@ -1,0 +1,303 @@
+// Band emission (ordered stream compaction) and the server-side average for MLMC-Top-k.
+//
+// emit: one sweep over every worker's gradient writes the band of the drawn level,
+//   { i : k_{l-1} < rank(i) <= k_l },  as (i, g_i / p_l) in ascending i  (Eq. 5 with g^0 = 0; Alg. 2 "Send").
+// Membership is decided from the two thresholds (Ta, ra), (Tb, rb) of the band; equal-key elements
+// are admitted by their index-ordered rank, so the running counts
+//   D  = #{ Tb < key <= Ta },  Ea = #{ key == Ta },  Eb = #{ key == Tb }
+// are carried across tiles with a decoupled look-back (tiles are handed out by a ticket counter, so
+// every predecessor of a running tile has already started; every wait is bounded).
+//
+// aggregate: the dense mean (1/M) sum_m g~_m (Alg. 2 "Server aggregates") tiled over the index
+// space; because every message is index-sorted, a tile's entries are one contiguous range per
+// worker; they are added into a shared-memory tile in worker order and the tile is written once.
+#include "common.cuh"
+
+namespace mlmc {
+
+namespace {
+
+constexpr unsigned kSpinLimit = 1u << 22;  // polls of ~100 ns each before a look-back gives up
+
+__device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) {
+    return *reinterpret_cast<const volatile uint32_t*>(p);
+}
+
+__device__ __forceinline__ void publish(TileRec* rec, uint32_t D, uint32_t Ea, uint32_t Eb) {
+    volatile TileRec* v = rec;
+    v->D = D;
+    v->Ea = Ea;
+    v->Eb = Eb;
+    __threadfence();
+    v->flag = 1u;
+}
+
+__device__ __forceinline__ uint32_t warp_sum(uint32_t x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+    return x;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kEmitThreads)
+emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker, unsigned total_tiles,
+            const EmitParams* __restrict__ emit, TileRec* tile_agg, TileRec* tile_inc, unsigned* tile_counter,
+            uint32_t* __restrict__ idx_out, float* __restrict__ val_out, int64_t capacity, int* status,
+            int* worker_err) {
+    using Tr = ElemTraits<T>;
+    constexpr int V = Tr::kVec;
+    constexpr int NV = kEmitItems / V;
+    __shared__ unsigned sh_ticket;
+    __shared__ unsigned long long sh_warp[kEmitThreads / 32];
+    __shared__ uint32_t sh_prefix[4];  // D, Ea, Eb, ok
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    while (true) {
+        if (threadIdx.x == 0) sh_ticket = atomicAdd(tile_counter, 1u);
+        __syncthreads();
+        const unsigned tile = sh_ticket;
+        __syncthreads();
+        if (tile >= total_tiles) break;
+        const int m = (int)(tile / (unsigned)tiles_per_worker);
+        const int t = (int)(tile % (unsigned)tiles_per_worker);
+        const EmitParams e = emit[m];
+        if (!e.enabled) continue;
+
+        // ---- load this thread's 16 consecutive elements
+        const T* row = g + (int64_t)m * ld;
+        const int64_t i0 = (int64_t)t * kEmitTile + (int64_t)threadIdx.x * kEmitItems;
+        uint32_t bits[kEmitItems];
+        uint32_t valid = 0;
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            const int64_t base = i0 + j * V;
+            if (base + V <= d) {
+                const uint4 q = __ldg(reinterpret_cast<const uint4*>(row + base));
+                if constexpr (V == 4) {
+                    bits[j * 4 + 0] = q.x; bits[j * 4 + 1] = q.y; bits[j * 4 + 2] = q.z; bits[j * 4 + 3] = q.w;
+                } else {
+                    bits[j * 8 + 0] = q.x & 0xFFFFu; bits[j * 8 + 1] = q.x >> 16;
+                    bits[j * 8 + 2] = q.y & 0xFFFFu; bits[j * 8 + 3] = q.y >> 16;
+                    bits[j * 8 + 4] = q.z & 0xFFFFu; bits[j * 8 + 5] = q.z >> 16;
+                    bits[j * 8 + 6] = q.w & 0xFFFFu; bits[j * 8 + 7] = q.w >> 16;
+                }
+                valid |= ((1u << V) - 1u) << (j * V);
+            } else {
+#pragma unroll
+                for (int c = 0; c < V; ++c) {
+                    bits[j * V + c] = 0;
+                    if (base + c < d) {
+                        if constexpr (V == 4)
+                            bits[j * V + c] = reinterpret_cast<const uint32_t*>(row)[base + c];
+                        else
+                            bits[j * V + c] = reinterpret_cast<const uint16_t*>(row)[base + c];
+                        valid |= 1u << (j * V + c);
+                    }
+                }
+            }
+        }
+
+        // ---- local counts, packed 21 bits each: D | Ea << 21 | Eb << 42
+        unsigned long long pack = 0;
+#pragma unroll
+        for (int i = 0; i < kEmitItems; ++i) {
+            const uint32_t key = Tr::key(bits[i]);
+            const bool ok = (valid >> i) & 1u;
+            const unsigned long long dD = (ok && key > e.Tb && key <= e.Ta) ? 1ull : 0ull;
+            const unsigned long long dA = (ok && key == e.Ta) ? 1ull : 0ull;
+            const unsigned long long dB = (ok && key == e.Tb) ? 1ull : 0ull;
+            pack += dD | (dA << 21) | (dB << 42);
+        }
+        // block exclusive scan of pack
+        unsigned long long inc = pack;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) sh_warp[warp] = inc;
+        __syncthreads();
+        unsigned long long warp_off = 0, block_total = 0;
+#pragma unroll
+        for (int w = 0; w < kEmitThreads / 32; ++w) {
+            const unsigned long long s = sh_warp[w];
+            if (w < warp) warp_off += s;
+            block_total += s;
+        }
+        const unsigned long long excl = inc - pack + warp_off;
+        const uint32_t aggD = (uint32_t)(block_total & 0x1FFFFFu);
+        const uint32_t aggA = (uint32_t)((block_total >> 21) & 0x1FFFFFu);
+        const uint32_t aggB = (uint32_t)((block_total >> 42) & 0x1FFFFFu);
+
+        // ---- decoupled look-back over this worker's earlier tiles (warp 0)
+        if (warp == 0) {
+            uint32_t pD = 0, pA = 0, pB = 0;
+            bool ok = true;
+            if (t > 0) {
+                if (lane == 0) publish(&tile_agg[tile], aggD, aggA, aggB);
+                const long long first = (long long)tile - t;  // first tile of this worker
+                long long look = (long long)tile - 1;
+                unsigned spins = 0;
+                while (true) {
+                    const long long at = look - lane;
+                    const bool real = at >= first;
+                    int st = real ? 0 : 2;  // positions before the worker's first tile count as a zero prefix
+                    while (true) {
+                        if (st == 0) {
+                            if (ld_volatile_u32(&tile_inc[at].flag)) st = 2;
+                            else if (ld_volatile_u32(&tile_agg[at].flag)) st = 1;
+                        }
+                        if (__all_sync(0xFFFFFFFFu, st != 0)) break;
+                        __nanosleep(100);
+                        const bool bail = (++spins > kSpinLimit) ||
+                                          ld_volatile_u32(reinterpret_cast<const uint32_t*>(status)) ==
+                                              (uint32_t)MLMC_ERR_TIMEOUT;
+                        if (__any_sync(0xFFFFFFFFu, bail)) {  // warp-uniform exit
+                            ok = false;
+                            break;
+                        }
+                    }
+                    if (!ok) break;
+                    __threadfence();
+                    uint32_t vD = 0, vA = 0, vB = 0;
+                    if (real) {
+                        const volatile TileRec* r = (st == 2) ? &tile_inc[at] : &tile_agg[at];
+                        vD = r->D; vA = r->Ea; vB = r->Eb;
+                    }
+                    const unsigned has_inc = __ballot_sync(0xFFFFFFFFu, st == 2);
+                    const int stop = has_inc ? (__ffs(has_inc) - 1) : 32;  // nearest predecessor with a full prefix
+                    const bool use = lane <= stop;
+                    pD += warp_sum(use ? vD : 0u);
+                    pA += warp_sum(use ? vA : 0u);
+                    pB += warp_sum(use ? vB : 0u);
+                    if (has_inc) break;
+                    look -= 32;
+                }
+                if (!ok) {
+                    set_status(status, MLMC_ERR_TIMEOUT);
+                    worker_err[m] = MLMC_ERR_TIMEOUT;
+                }
+            }
+            if (lane == 0) {
+                publish(&tile_inc[tile], pD + aggD, pA + aggA, pB + aggB);  // also after a timeout, so successors move on
+                sh_prefix[0] = pD; sh_prefix[1] = pA; sh_prefix[2] = pB; sh_prefix[3] = ok ? 1u : 0u;
+            }
+        }
+        __syncthreads();
+        const bool ok = sh_prefix[3] != 0;
+        uint32_t rD = sh_prefix[0] + (uint32_t)(excl & 0x1FFFFFu);
+        uint32_t rA = sh_prefix[1] + (uint32_t)((excl >> 21) & 0x1FFFFFu);
+        uint32_t rB = sh_prefix[2] + (uint32_t)((excl >> 42) & 0x1FFFFFu);
+
+        // ---- self-check on the worker's last tile: the band has exactly k_l - k_{l-1} entries
+        if (t == tiles_per_worker - 1 && threadIdx.x == 0 && ok) {
+            const uint32_t tD = sh_prefix[0] + aggD, tA = sh_prefix[1] + aggA, tB = sh_prefix[2] + aggB;
+            const uint32_t total = tD + min(tB, e.rb) - min(tA, e.ra);
+            if (total != e.expect) set_status(status, MLMC_ERR_INTERNAL);
+        }
+
+        // ---- write the band entries at their global positions
+        if (ok && (aggD | aggA | aggB)) {
+            uint32_t* idx_w = idx_out + (int64_t)m * capacity;
+            float* val_w = val_out + (int64_t)m * capacity;
+#pragma unroll
+            for (int i = 0; i < kEmitItems; ++i) {
+                const uint32_t key = Tr::key(bits[i]);
+                const bool okv = (valid >> i) & 1u;
+                const bool eqA = okv && key == e.Ta, eqB = okv && key == e.Tb;
+                const bool insA = okv && (key > e.Ta || (eqA && rA < e.ra));   // tie rank rA + 1 <= ra
+                const bool insB = okv && (key > e.Tb || (eqB && rB < e.rb));
+                if (insB && !insA) {
+                    const uint32_t pos = rD + min(rB, e.rb) - min(rA, e.ra);
+                    if ((int64_t)pos < capacity) {
+                        idx_w[pos] = (uint32_t)(i0 + i);
+                        val_w[pos] = (float)((double)Tr::value(bits[i]) * e.inv_p);
+                    }
+                }
+                rD += (okv && key > e.Tb && key <= e.Ta) ? 1u : 0u;
+                rA += eqA ? 1u : 0u;
+                rB += eqB ? 1u : 0u;
+            }
+        }
+    }
+}
+
+// offsets[m][t] = first message entry of worker m whose index is >= t * kAggTile  (t = 0..ntiles)
+__global__ void agg_offsets_kernel(const uint32_t* __restrict__ idx, const int64_t* __restrict__ count,
+                                   const int32_t* __restrict__ level, int64_t capacity, int M, int ntiles,
+                                   uint32_t* __restrict__ offsets) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)M * (ntiles + 1)) return;
+    const int m = (int)(i / (ntiles + 1)), t = (int)(i % (ntiles + 1));
+    const int64_t n = (level[m] < 0) ? 0 : count[m];
+    const uint32_t* a = idx + (int64_t)m * capacity;
+    const uint64_t target = (uint64_t)t * kAggTile;
+    int64_t lo = 0, hi = n;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((uint64_t)a[mid] < target) lo = mid + 1; else hi = mid;
+    }
+    offsets[i] = (uint32_t)lo;
+}
+
+__global__ void __launch_bounds__(256)
+aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict__ val, int64_t capacity, int M,
+                      int64_t d, int ntiles, const uint32_t* __restrict__ offsets, float* __restrict__ out) {
+    __shared__ float acc[kAggTile];
+    const float fM = (float)M;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const int64_t base = (int64_t)t * kAggTile;
+        for (int i = threadIdx.x; i < kAggTile; i += blockDim.x) acc[i] = 0.0f;
+        __syncthreads();
+        for (int m = 0; m < M; ++m) {  // fixed worker order: reproducible fp32 sums
+            const uint32_t o0 = offsets[(int64_t)m * (ntiles + 1) + t];
+            const uint32_t o1 = offsets[(int64_t)m * (ntiles + 1) + t + 1];
+            if (o1 > o0) {
+                const uint32_t* a = idx + (int64_t)m * capacity;
+                const float* v = val + (int64_t)m * capacity;
+                for (uint32_t j = o0 + threadIdx.x; j < o1; j += blockDim.x)
+                    acc[a[j] - (uint32_t)base] += v[j];  // indices are unique within a worker
+                __syncthreads();
+            }
+        }
+        for (int i = threadIdx.x; i < kAggTile; i += blockDim.x)
+            if (base + i < d) out[base + i] = acc[i] / fM;
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const mlmc_topk_msgs& out,
+                 cudaStream_t s) {
+    const int tpw = (int)((d + kEmitTile - 1) / kEmitTile);
+    const unsigned total = (unsigned)tpw * (unsigned)M;
+    cudaMemsetAsync(ws.tile_agg, 0, (size_t)total * sizeof(TileRec), s);
+    cudaMemsetAsync(ws.tile_inc, 0, (size_t)total * sizeof(TileRec), s);
+    cudaMemsetAsync(ws.tile_counter, 0, sizeof(unsigned), s);
+    unsigned grid = (unsigned)ws.sm_count * 8u;
+    if (grid > total) grid = total;
+    if (dtype == MLMC_BF16)
+        emit_kernel<bf16_t><<<grid, kEmitThreads, 0, s>>>(static_cast<const bf16_t*>(g), d, ld, tpw, total, ws.emit,
+                                                         ws.tile_agg, ws.tile_inc, ws.tile_counter, out.idx, out.val,
+                                                         out.capacity, ws.status, ws.worker_err);
+    else
+        emit_kernel<float><<<grid, kEmitThreads, 0, s>>>(static_cast<const float*>(g), d, ld, tpw, total, ws.emit,
+                                                        ws.tile_agg, ws.tile_inc, ws.tile_counter, out.idx, out.val,
+                                                        out.capacity, ws.status, ws.worker_err);
+    ws.launches++;
+}
+
+void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int64_t d, float* out, cudaStream_t s) {
+    const int ntiles = (int)((d + kAggTile - 1) / kAggTile);
+    const int64_t n_off = (int64_t)M * (ntiles + 1);
+    agg_offsets_kernel<<<(unsigned)((n_off + 255) / 256), 256, 0, s>>>(msgs.idx, msgs.count, msgs.level, msgs.capacity,
+                                                                       M, ntiles, ws.agg_offsets);
+    ws.launches++;
+    int grid = ws.sm_count * 8;
+    if (grid > ntiles) grid = ntiles;
+    aggregate_topk_kernel<<<grid, 256, 0, s>>>(msgs.idx, msgs.val, msgs.capacity, M, d, ntiles, ws.agg_offsets, out);
+    ws.launches++;
+}
+
+}  // namespace mlmc

@@ -1,0 +1,656 @@
+// Threshold selection, band norms, level probabilities and the level draw for MLMC-Top-k.
+//
+// The residual C^l(g) - C^{l-1}(g) of Top-k is the band of ranks (k_{l-1}, k_l] of the total order
+// (|g| descending, index ascending) (Sec. 3.2).  A band is described by two thresholds: for rank k,
+// T = key of the rank-k element, c = #{key > T}, n = #{key == T}, r = k - c = how many of the
+// equal-key elements (in index order) are inside Top-k.  Thresholds come from an MSD radix select
+// on the magnitude key: a 2^15-bin histogram of the leading digit for all queries at once, then two
+// 8-bit digit passes restricted to the boundary bins (fp32 only; a bf16 key is its leading digit).
+#include "common.cuh"
+
+namespace mlmc {
+
+namespace {
+
+constexpr int kHistThreads = 1024;
+constexpr int kResolveThreads = 1024;
+
+// -------------------------------------------------------------------------------------------
+// queries
+// -------------------------------------------------------------------------------------------
+// Adaptive: every level boundary k_0..k_{L-2} is a query.  Fixed p: the level is drawn first
+// (it does not depend on the data), and only the two boundaries of its band are live.
+__global__ void init_queries_kernel(Query* queries, const int64_t* k, int L, int64_t d, const EmitParams* emit,
+                                    int fixed) {
+    const int m = blockIdx.x;
+    const int j = threadIdx.x;
+    if (j >= L - 1) return;
+    Query q = {};
+    const int64_t kj = k[j];
+    q.k = (uint32_t)kj;
+    q.slot = kNoSlot;
+    q.trivial = (kj <= 0) ? 1u : (kj >= d ? 2u : 0u);
+    if (fixed) {
+        const int lv = emit[m].level;
+        if (j != lv && j != lv - 1) q.trivial = 3u;
+    }
+    if (q.trivial == 1u || q.trivial == 3u) {
+        q.T = kKeyNone;
+    } else if (q.trivial == 2u) {
+        q.T = 0u;
+        q.r = 0xFFFFFFFFu;
+    }
+    queries[m * kMaxQueries + j] = q;
+}
+
+// cdf in ascending l; the last level with p > 0 and everything after it has cdf 1; l* = min{l : u < cdf_l}.
+__device__ int draw_level(const double* p, int L, double u) {
+    int j_last = -1;
+    for (int j = 0; j < L; ++j)
+        if (p[j] > 0.0) j_last = j;
+    double c = 0.0;
+    for (int j = 0; j < L; ++j) {
+        c += p[j];
+        const double cdf = (j >= j_last) ? 1.0 : c;
+        if (u < cdf) return j;
+    }
+    return 0;
+}
+
+__global__ void draw_fixed_kernel(const double* p_fixed, int L, uint64_t seed, uint64_t step, double* p_all,
+                                  double* u_dev, EmitParams* emit, int M) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= M) return;
+    const double u = counter_uniform(seed, step, (uint64_t)m);
+    u_dev[m] = u;
+    for (int l = 0; l < L; ++l) p_all[m * kMaxLevels + l] = p_fixed[l];
+    emit[m].level = draw_level(p_fixed, L, u);
+}
+
+__global__ void uniforms_kernel(double* u_dev, int M, uint64_t seed, uint64_t step) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < M) u_dev[m] = counter_uniform(seed, step, (uint64_t)m);
+}
+
+// -------------------------------------------------------------------------------------------
+// sweep 1: leading-digit histogram of every worker (shared-memory counts, flushed with atomics)
+// -------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kHistThreads, 1)
+hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restrict__ hist1, int* status,
+             int* worker_err) {
+    extern __shared__ uint32_t sh_hist[];
+    using Tr = ElemTraits<T>;
+    const int m = blockIdx.y;
+    for (int b = threadIdx.x; b < kBins1; b += blockDim.x) sh_hist[b] = 0;
+    __syncthreads();
+    const T* row = g + (int64_t)m * ld;
+    int64_t v0, v1;
+    block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
+    bool bad = false;
+#pragma unroll 4
+    for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+        for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) {
+            const uint32_t key = Tr::key(bits);
+            bad |= (key >= Tr::kInfKey);
+            atomicAdd(&sh_hist[key >> Tr::kShift1], 1u);
+        });
+    }
+    if (bad) {
+        worker_err[m] = MLMC_ERR_NONFINITE;
+        set_status(status, MLMC_ERR_NONFINITE);
+    }
+    __syncthreads();
+    uint32_t* out = hist1 + (int64_t)m * kBins1;
+    for (int b = threadIdx.x; b < kBins1; b += blockDim.x) {
+        const uint32_t c = sh_hist[b];
+        if (c) atomicAdd(&out[b], c);
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+// block-level helpers for the per-worker resolve kernels
+// -------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t x) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+        if (lane >= o) x += y;
+    }
+    return x;
+}
+
+// Exclusive prefix over threads in DESCENDING thread order (thread t gets the sum of threads > t).
+__device__ uint32_t block_exclusive_suffix(uint32_t x, uint32_t* sh_warp /* [32] */) {
+    const int nt = blockDim.x;
+    const int rt = nt - 1 - threadIdx.x;  // reversed thread index
+    // emulate a forward scan over reversed indices by exchanging through shared memory
+    __shared__ uint32_t sh_x[kResolveThreads];
+    sh_x[rt] = x;
+    __syncthreads();
+    const uint32_t mine = sh_x[threadIdx.x];  // value of reversed position threadIdx.x
+    const uint32_t inc = warp_inclusive_sum(mine);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 31) sh_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t w = (lane < (nt >> 5)) ? sh_warp[lane] : 0u;
+        const uint32_t winc = warp_inclusive_sum(w);
+        sh_warp[lane] = winc - w;
+    }
+    __syncthreads();
+    const uint32_t exc = inc - mine + sh_warp[warp];  // exclusive prefix at reversed position threadIdx.x
+    __syncthreads();
+    sh_x[threadIdx.x] = exc;
+    __syncthreads();
+    const uint32_t res = sh_x[rt];
+    __syncthreads();
+    return res;
+}
+
+// Assigns histogram slots to live queries: queries whose fixed prefix (>> shift) agree share a slot.
+__device__ void assign_slots(Query* q, int nq, int shift) {
+    int next = 0;
+    for (int j = 0; j < nq; ++j) {
+        if (q[j].trivial) continue;
+        int s = -1;
+        for (int i = 0; i < j; ++i)
+            if (!q[i].trivial && (q[i].prefix >> shift) == (q[j].prefix >> shift)) {
+                s = (int)q[i].slot;
+                break;
+            }
+        q[j].slot = (s >= 0) ? (uint32_t)s : (uint32_t)next++;
+    }
+}
+
+// After sweep 1: suffix sums of the leading-digit histogram in place (S[b] = #{digit >= b}), then
+// every live query descends into its bin.  For bf16 the digit is the whole key, so the query is resolved.
+__global__ void __launch_bounds__(kResolveThreads, 1)
+resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is_bf16, const int* worker_err) {
+    __shared__ uint32_t sh_warp[32];
+    const int m = blockIdx.x;
+    uint32_t* S = hist1 + (int64_t)m * kBins1;
+    Query* q = queries + m * kMaxQueries;
+    constexpr int per = kBins1 / kResolveThreads;  // 32 bins per thread
+    const int b0 = threadIdx.x * per;
+    uint32_t local = 0;
+    for (int i = 0; i < per; ++i) local += S[b0 + i];
+    uint32_t above = block_exclusive_suffix(local, sh_warp);
+    for (int i = per - 1; i >= 0; --i) {
+        above += S[b0 + i];
+        S[b0 + i] = above;
+    }
+    __syncthreads();
+    if (worker_err[m]) return;
+    if (threadIdx.x < nq && !q[threadIdx.x].trivial) {
+        Query& qq = q[threadIdx.x];
+        int lo = 0, hi = kBins1 - 1;  // largest b with S[b] >= k  (S[0] = d >= k)
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (S[mid] >= qq.k) lo = mid; else hi = mid - 1;
+        }
+        const uint32_t ab = (lo == kBins1 - 1) ? 0u : S[lo + 1];
+        if (is_bf16) {
+            qq.T = (uint32_t)lo;
+            qq.c = ab;
+            qq.n = S[lo] - ab;
+            qq.r = qq.k - ab;
+        } else {
+            qq.prefix = (uint32_t)lo << 16;
+            qq.rem = qq.k - ab;
+        }
+    }
+    __syncthreads();
+    if (!is_bf16 && threadIdx.x == 0) {
+        assign_slots(q, nq, 16);
+        for (int j = 0; j < nq; ++j)
+            if (!q[j].trivial) table1[(int64_t)m * kBins1 + (q[j].prefix >> 16)] = (uint8_t)q[j].slot;
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+// digit passes 2 and 3 (fp32): histogram of the next 8 bits over the elements of the boundary bins
+// -------------------------------------------------------------------------------------------
+template <int PASS>
+__global__ void __launch_bounds__(kSweepThreads)
+masked_pass_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table1,
+                   const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err) {
+    extern __shared__ uint8_t sh_raw[];
+    uint32_t* sh_hist = reinterpret_cast<uint32_t*>(sh_raw);                        // [32][256]
+    uint8_t* sh_table = sh_raw + kMaxQueries * kBins23 * sizeof(uint32_t);          // [32768]
+    uint8_t* sh_map = sh_table + kBins1;                                            // [32][256] (pass 3)
+    const int m = blockIdx.y;
+    if (worker_err[m]) return;
+    for (int i = threadIdx.x; i < kMaxQueries * kBins23; i += blockDim.x) sh_hist[i] = 0;
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(table1 + (int64_t)m * kBins1);
+        uint4* dst = reinterpret_cast<uint4*>(sh_table);
+        for (int i = threadIdx.x; i < kBins1 / 16; i += blockDim.x) dst[i] = src[i];
+        if (PASS == 3) {
+            const uint4* s2 = reinterpret_cast<const uint4*>(map2 + (int64_t)m * kMaxQueries * kBins23);
+            uint4* d2 = reinterpret_cast<uint4*>(sh_map);
+            for (int i = threadIdx.x; i < kMaxQueries * kBins23 / 16; i += blockDim.x) d2[i] = s2[i];
+        }
+    }
+    __syncthreads();
+    const float* row = g + (int64_t)m * ld;
+    int64_t v0, v1;
+    block_vector_range(d, 4, blockIdx.x, gridDim.x, &v0, &v1);
+#pragma unroll 4
+    for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+        for_each_in_vector<float>(row, v, d, [&](int64_t, uint32_t bits) {
+            const uint32_t key = bits & 0x7FFFFFFFu;
+            const uint32_t s2 = sh_table[key >> 16];
+            if (s2 != kNoSlot) {
+                if (PASS == 2) {
+                    atomicAdd(&sh_hist[s2 * kBins23 + ((key >> 8) & 0xFFu)], 1u);
+                } else {
+                    const uint32_t s3 = sh_map[s2 * kBins23 + ((key >> 8) & 0xFFu)];
+                    if (s3 != kNoSlot) atomicAdd(&sh_hist[s3 * kBins23 + (key & 0xFFu)], 1u);
+                }
+            }
+        });
+    }
+    __syncthreads();
+    uint32_t* out = hist_out + (int64_t)m * kMaxQueries * kBins23;
+    for (int i = threadIdx.x; i < kMaxQueries * kBins23; i += blockDim.x) {
+        const uint32_t c = sh_hist[i];
+        if (c) atomicAdd(&out[i], c);
+    }
+}
+
+// One warp per query walks its 256-bin histogram from the top digit down.
+template <int PASS>
+__global__ void __launch_bounds__(kResolveThreads, 1)
+resolve23_kernel(const uint32_t* hist, Query* queries, uint8_t* map2, int nq, const int* worker_err) {
+    const int m = blockIdx.x;
+    if (worker_err[m]) return;
+    Query* q = queries + m * kMaxQueries;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp < nq && !q[warp].trivial) {
+        Query& qq = q[warp];
+        const uint32_t* h = hist + ((int64_t)m * kMaxQueries + qq.slot) * kBins23;
+        // lane 0 owns the top 8 digits (255..248), lane 31 the bottom 8
+        uint32_t cnt[8], local = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            cnt[i] = h[255 - (lane * 8 + i)];
+            local += cnt[i];
+        }
+        const uint32_t inc = warp_inclusive_sum(local);
+        const uint32_t rem = qq.rem;
+        const bool mine = (inc >= rem) && (inc - local < rem);
+        if (mine) {
+            uint32_t above = inc - local;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (above + cnt[i] >= rem) {
+                    const uint32_t digit = 255u - (uint32_t)(lane * 8 + i);
+                    if (PASS == 2) {
+                        qq.prefix |= digit << 8;
+                        qq.rem = rem - above;
+                    } else {
+                        qq.T = qq.prefix | digit;
+                        qq.r = rem - above;
+                        qq.n = cnt[i];
+                        qq.c = qq.k - qq.r;
+                    }
+                    break;
+                }
+                above += cnt[i];
+            }
+        }
+    }
+    __syncthreads();
+    if (PASS == 2 && threadIdx.x == 0) {
+        // remember the pass-2 slot of each query before the slots are reassigned for pass 3
+        uint32_t slot2[kMaxQueries];
+        for (int j = 0; j < nq; ++j) slot2[j] = q[j].slot;
+        assign_slots(q, nq, 8);
+        for (int j = 0; j < nq; ++j)
+            if (!q[j].trivial)
+                map2[((int64_t)m * kMaxQueries + slot2[j]) * kBins23 + ((q[j].prefix >> 8) & 0xFFu)] = (uint8_t)q[j].slot;
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+// band norms (adaptive): sum of g^2 over the open key intervals between consecutive thresholds
+// -------------------------------------------------------------------------------------------
+// Element with key x belongs to open interval b = #{ l : T_l > x } unless x equals a threshold
+// (equal-key elements are split between bands by rank; their energy is added from the counts).
+// Every thread owns a private fp64 accumulator per interval in shared memory: no atomics, and a
+// fixed reduction order, so the sums are reproducible.
+__global__ void __launch_bounds__(kSweepThreads)
+norm_sweep_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const Query* __restrict__ queries, int L,
+                  double* __restrict__ band_partial, int norm_ctas, const int* worker_err) {
+    extern __shared__ double sh_acc[];  // [L][blockDim]
+    __shared__ uint32_t sh_thr[kMaxQueries];
+    const int m = blockIdx.y;
+    if (worker_err[m]) return;
+    const int nt = blockDim.x;
+    for (int i = threadIdx.x; i < L * nt; i += nt) sh_acc[i] = 0.0;
+    if (threadIdx.x < kMaxQueries)
+        sh_thr[threadIdx.x] = (threadIdx.x < L - 1) ? queries[m * kMaxQueries + threadIdx.x].T : 0u;
+    __syncthreads();
+    const float* row = g + (int64_t)m * ld;
+    int64_t v0, v1;
+    block_vector_range(d, 4, blockIdx.x, gridDim.x, &v0, &v1);
+    const int nthr = L - 1;
+#pragma unroll 2
+    for (int64_t v = v0 + threadIdx.x; v < v1; v += nt) {
+        for_each_in_vector<float>(row, v, d, [&](int64_t, uint32_t bits) {
+            const uint32_t key = bits & 0x7FFFFFFFu;
+            // thresholds are descending: b = first index with T_b <= key
+            int lo = 0, hi = nthr;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (sh_thr[mid] > key) lo = mid + 1; else hi = mid;
+            }
+            if (lo == nthr || sh_thr[lo] != key) {
+                const double x = (double)__uint_as_float(key);
+                double* a = &sh_acc[lo * nt + threadIdx.x];
+                *a = fma(x, x, *a);
+            }
+        });
+    }
+    __syncthreads();
+    // fixed-order tree reduction per interval
+    for (int l = 0; l < L; ++l) {
+        double* a = sh_acc + l * nt;
+        for (int s = nt >> 1; s > 0; s >>= 1) {
+            if (threadIdx.x < s) a[threadIdx.x] += a[threadIdx.x + s];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) band_partial[((int64_t)m * norm_ctas + blockIdx.x) * kMaxLevels + l] = a[0];
+    }
+}
+
+// bf16: every key is a histogram bin, so the open-interval sums follow from the counts exactly.
+__global__ void __launch_bounds__(kResolveThreads, 1)
+norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query* queries, int L,
+                           double* band_partial, int norm_ctas, const int* worker_err) {
+    __shared__ double sh_red[kResolveThreads];
+    __shared__ uint32_t sh_thr[kMaxQueries];
+    const int m = blockIdx.x;
+    if (worker_err[m]) return;
+    const uint32_t* S = hist1 + (int64_t)m * kBins1;
+    if (threadIdx.x < kMaxQueries)
+        sh_thr[threadIdx.x] = (threadIdx.x < L - 1) ? queries[m * kMaxQueries + threadIdx.x].T : 0u;
+    __syncthreads();
+    constexpr int per = kBins1 / kResolveThreads;
+    for (int l = 0; l < L; ++l) {
+        // open interval l: T_l < key < T_{l-1}   (T_{-1} = +inf, T_{L-1} = -1: everything below)
+        const uint32_t hi = (l == 0) ? 0xFFFFFFFFu : sh_thr[l - 1];
+        const int64_t lo = (l == L - 1) ? -1 : (int64_t)sh_thr[l];
+        double acc = 0.0;
+        for (int i = 0; i < per; ++i) {
+            const uint32_t key = threadIdx.x * per + i;
+            if ((int64_t)key > lo && key < hi) {
+                const uint32_t cnt = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
+                const double x = (double)__uint_as_float(key << 16);
+                acc = fma((double)cnt, x * x, acc);
+            }
+        }
+        sh_red[threadIdx.x] = acc;
+        __syncthreads();
+        for (int s = kResolveThreads >> 1; s > 0; s >>= 1) {
+            if (threadIdx.x < s) sh_red[threadIdx.x] += sh_red[threadIdx.x + s];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) band_partial[((int64_t)m * norm_ctas) * kMaxLevels + l] = sh_red[0];
+        __syncthreads();
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+// probabilities, draw, emit parameters
+// -------------------------------------------------------------------------------------------
+__device__ void fill_emit(int m, int level, double p_sel, const Query* q, const int64_t* k, int L, int64_t d,
+                          EmitParams* emit, int64_t* out_count, int32_t* out_level, double* out_p_sel,
+                          int64_t capacity, int* status, int* worker_err) {
+    EmitParams e = {};
+    e.level = level;
+    if (level == 0) {
+        e.Ta = kKeyNone;
+        e.ra = 0;
+    } else {
+        e.Ta = q[level - 1].T;
+        e.ra = q[level - 1].r;
+    }
+    if (level == L - 1) {
+        e.Tb = 0u;
+        e.rb = 0xFFFFFFFFu;
+    } else {
+        e.Tb = q[level].T;
+        e.rb = q[level].r;
+    }
+    e.inv_p = (p_sel > 0.0) ? 1.0 / p_sel : 0.0;
+    const int64_t lo = level ? k[level - 1] : 0;
+    e.expect = (uint32_t)(k[level] - lo);
+    e.enabled = 1;
+    if ((int64_t)e.expect > capacity) {
+        e.enabled = 0;
+        worker_err[m] = MLMC_ERR_CAPACITY;
+        set_status(status, MLMC_ERR_CAPACITY);
+    }
+    emit[m] = e;
+    out_count[m] = e.enabled ? (int64_t)e.expect : 0;
+    out_level[m] = e.enabled ? level : -1;
+    out_p_sel[m] = p_sel;
+}
+
+__device__ void fail_worker(int m, EmitParams* emit, int64_t* out_count, int32_t* out_level, double* out_p_sel) {
+    EmitParams e = {};
+    e.level = -1;
+    emit[m] = e;
+    if (out_count) out_count[m] = 0;
+    if (out_level) out_level[m] = -1;
+    if (out_p_sel) out_p_sel[m] = 0.0;
+}
+
+// One block per worker.  Adaptive: E_l = open-interval sum + sum over distinct threshold keys K of
+// |ranks of K  intersect  (k_{l-1}, k_l]| * val(K)^2;  Delta_l = sqrt(E_l);  p_l = Delta_l / sum Delta
+// (Lemma 3.4).  Then the level draw and the two thresholds of the drawn band.
+__global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L, int64_t d, int is_bf16,
+                                  const double* band_partial, int n_partials, int norm_ctas, int adaptive,
+                                  uint64_t seed, uint64_t step, double* p_all, double* delta_all, double* u_dev,
+                                  EmitParams* emit, int64_t* out_count, int32_t* out_level, double* out_p_sel,
+                                  int64_t capacity, int* status, int* worker_err, int want_emit) {
+    __shared__ double sh_delta[kMaxLevels];
+    __shared__ double sh_p[kMaxLevels];
+    const int m = blockIdx.x;
+    const Query* q = queries + m * kMaxQueries;
+    if (worker_err[m]) {
+        if (threadIdx.x == 0 && want_emit) fail_worker(m, emit, out_count, out_level, out_p_sel);
+        return;
+    }
+    const int l = threadIdx.x;
+    if (adaptive && l < L) {
+        double E = 0.0;
+        for (int c = 0; c < n_partials; ++c) E += band_partial[((int64_t)m * norm_ctas + c) * kMaxLevels + l];
+        const int64_t lo = l ? k[l - 1] : 0, hi = k[l];
+        for (int j = 0; j < L - 1; ++j) {
+            if (q[j].trivial) continue;
+            bool dup = false;
+            for (int i = 0; i < j; ++i) dup |= (!q[i].trivial && q[i].T == q[j].T);
+            if (dup) continue;
+            const int64_t c0 = q[j].c, c1 = c0 + (int64_t)q[j].n;
+            const int64_t ov = min(c1, hi) - max(c0, lo);
+            if (ov > 0) {
+                const uint32_t bits = is_bf16 ? (q[j].T << 16) : q[j].T;
+                const double x = (double)__uint_as_float(bits);
+                E = fma((double)ov, x * x, E);
+            }
+        }
+        sh_delta[l] = sqrt(E);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double p_sel;
+        int level;
+        if (adaptive) {
+            double s = 0.0;
+            for (int i = 0; i < L; ++i) s += sh_delta[i];
+            for (int i = 0; i < L; ++i) {
+                sh_p[i] = (s > 0.0) ? sh_delta[i] / s : (i == 0 ? 1.0 : 0.0);
+                p_all[m * kMaxLevels + i] = sh_p[i];
+                delta_all[m * kMaxLevels + i] = sh_delta[i];
+            }
+            const double u = counter_uniform(seed, step, (uint64_t)m);
+            u_dev[m] = u;
+            level = draw_level(sh_p, L, u);
+            p_sel = sh_p[level];
+        } else {
+            level = emit[m].level;  // drawn before the sweeps
+            p_sel = p_all[m * kMaxLevels + level];
+        }
+        if (want_emit)
+            fill_emit(m, level, p_sel, q, k, L, d, emit, out_count, out_level, out_p_sel, capacity, status, worker_err);
+    }
+}
+
+__global__ void copy_probs_kernel(const double* p_all, const double* delta_all, const double* p_fixed, int M, int L,
+                                  double* p_out, double* delta_out, const int* worker_err) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M * L) return;
+    const int m = i / L, l = i % L;
+    const bool bad = worker_err[m] != 0;
+    if (p_out) p_out[i] = p_fixed ? p_fixed[l] : (bad ? 0.0 : p_all[m * kMaxLevels + l]);
+    if (delta_out) delta_out[i] = bad ? 0.0 : delta_all[m * kMaxLevels + l];
+}
+
+int blocks_per_worker(const Workspace& ws, int64_t d, int vec, int threads, int M, int waves) {
+    const int64_t nvec = (d + vec - 1) / vec;
+    const int64_t by_work = (nvec + (int64_t)threads * 4 - 1) / ((int64_t)threads * 4);
+    int64_t by_sm = ((int64_t)ws.sm_count * waves + M - 1) / M;
+    if (by_sm < 1) by_sm = 1;
+    int64_t nb = by_work < by_sm ? by_work : by_sm;
+    return (int)(nb < 1 ? 1 : nb);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------------
+void launch_init_queries_adaptive(Workspace& ws, int M, int L, int64_t d, cudaStream_t s) {
+    if (L > 1) {
+        init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 0);
+        ws.launches++;
+    }
+}
+
+void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, cudaStream_t s) {
+    draw_fixed_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.p_fixed, L, seed, step, ws.p_all, ws.u_dev, ws.emit, M);
+    ws.launches++;
+    if (L > 1) {
+        init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 1);
+        ws.launches++;
+    }
+}
+
+void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStream_t s) {
+    uniforms_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.u_dev, M, seed, step);
+    ws.launches++;
+}
+
+void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
+    cudaMemsetAsync(ws.hist1, 0, (size_t)M * kBins1 * sizeof(uint32_t), s);
+    const size_t smem = kBins1 * sizeof(uint32_t);
+    if (dtype == MLMC_BF16) {
+        const int nb = blocks_per_worker(ws, d, 8, kHistThreads, M, 2);
+        hist1_kernel<bf16_t><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const bf16_t*>(g), d, ld, ws.hist1,
+                                                                     ws.status, ws.worker_err);
+    } else {
+        const int nb = blocks_per_worker(ws, d, 4, kHistThreads, M, 2);
+        hist1_kernel<float><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.hist1,
+                                                                    ws.status, ws.worker_err);
+    }
+    ws.launches++;
+}
+
+void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
+    if (dtype != MLMC_BF16) cudaMemsetAsync(ws.table1, 0xFF, (size_t)M * kBins1, s);
+    resolve1_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, ws.table1, L - 1, dtype == MLMC_BF16,
+                                                  ws.worker_err);
+    ws.launches++;
+}
+
+void launch_masked_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s) {
+    const size_t hist_bytes = (size_t)M * kMaxQueries * kBins23 * sizeof(uint32_t);
+    const size_t smem = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
+    const int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 6);
+    if (pass == 2) {
+        cudaMemsetAsync(ws.hist2, 0, hist_bytes, s);
+        cudaMemsetAsync(ws.map2, 0xFF, (size_t)M * kMaxQueries * kBins23, s);
+        masked_pass_kernel<2><<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.table1,
+                                                                       ws.map2, ws.hist2, ws.worker_err);
+    } else {
+        cudaMemsetAsync(ws.hist3, 0, hist_bytes, s);
+        masked_pass_kernel<3><<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.table1,
+                                                                       ws.map2, ws.hist3, ws.worker_err);
+    }
+    ws.launches++;
+}
+
+void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
+    if (pass == 2)
+        resolve23_kernel<2><<<M, kResolveThreads, 0, s>>>(ws.hist2, ws.queries, ws.map2, L - 1, ws.worker_err);
+    else
+        resolve23_kernel<3><<<M, kResolveThreads, 0, s>>>(ws.hist3, ws.queries, ws.map2, L - 1, ws.worker_err);
+    ws.launches++;
+}
+
+void launch_norm_sweep(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
+    int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 4);
+    if (nb > ws.norm_ctas) nb = ws.norm_ctas;
+    const size_t smem = (size_t)L * kSweepThreads * sizeof(double);
+    cudaMemsetAsync(ws.band_partial, 0, (size_t)M * ws.norm_ctas * kMaxLevels * sizeof(double), s);
+    norm_sweep_kernel<<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.queries, L,
+                                                               ws.band_partial, ws.norm_ctas, ws.worker_err);
+    ws.launches++;
+}
+
+void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s) {
+    norm_from_hist_bf16_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, L, ws.band_partial, ws.norm_ctas,
+                                                             ws.worker_err);
+    ws.launches++;
+}
+
+void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool adaptive, bool want_emit,
+                       uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, cudaStream_t s) {
+    const int n_partials = (dtype == MLMC_BF16) ? 1 : ws.norm_ctas;
+    probs_draw_kernel<<<M, kMaxLevels, 0, s>>>(
+        ws.queries, ws.k_dev, L, d, dtype == MLMC_BF16, ws.band_partial, n_partials, ws.norm_ctas, adaptive ? 1 : 0,
+        seed, step, ws.p_all, ws.delta_all, ws.u_dev, ws.emit, out ? out->count : nullptr, out ? out->level : nullptr,
+        out ? out->p_sel : nullptr, out ? out->capacity : 0, ws.status, ws.worker_err, want_emit ? 1 : 0);
+    ws.launches++;
+}
+
+void launch_copy_probs(Workspace& ws, int M, int L, const double* p_fixed, double* p_out, double* delta_out,
+                       cudaStream_t s) {
+    copy_probs_kernel<<<(M * L + 127) / 128, 128, 0, s>>>(ws.p_all, ws.delta_all, p_fixed, M, L, p_out, delta_out,
+                                                          ws.worker_err);
+    ws.launches++;
+}
+
+int configure_select_kernels() {
+    cudaError_t e = cudaFuncSetAttribute(hist1_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(kBins1 * sizeof(uint32_t)));
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    e = cudaFuncSetAttribute(hist1_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kBins1 * sizeof(uint32_t)));
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    const int smem_masked = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
+    e = cudaFuncSetAttribute(masked_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_masked);
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    e = cudaFuncSetAttribute(masked_pass_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_masked);
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    e = cudaFuncSetAttribute(norm_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kMaxLevels * kSweepThreads * sizeof(double)));
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    return MLMC_OK;
+}
+
+}  // namespace mlmc
