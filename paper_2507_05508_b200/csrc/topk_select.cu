@@ -388,8 +388,10 @@ norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query*
             const uint32_t key = threadIdx.x * per + i;
             if ((int64_t)key > lo && key < hi) {
                 const uint32_t cnt = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
-                const double x = (double)__uint_as_float(key << 16);
-                acc = fma((double)cnt, x * x, acc);
+                if (cnt) {  // empty bins include the Inf/NaN encodings, whose value must not enter the sum
+                    const double x = (double)__uint_as_float(key << 16);
+                    acc = fma((double)cnt, x * x, acc);
+                }
             }
         }
         sh_red[threadIdx.x] = acc;
