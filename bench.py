@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the MLMC compress+aggregate hot path.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5a] [--impl reference]
+
+One step = mlmc_compress_* on all M workers + mlmc_aggregate into the dense mean, on one batch of
+synthetic gradients already resident in HBM.  `value` is gradient GB/s = M*d*sizeof(T) / step time,
+summed over ranks (ranks are independent replicas: the path has no inter-GPU exchange).
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "MLMC compress+aggregate gradient GB/s per step (1 B200); fraction of HBM peak"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic per launch of each sweep kernel relative to its algorithmic bytes, from the ncu captures
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same
+# kernel; traffic grows in proportion to the elements swept).  None = not captured yet.
+NCU_TRAFFIC_RATIO = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c5a", choices=["c1", "c2", "c3", "c4", "c5a", "c5b"])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def elem_size(w):
+    return 2 if w.dtype == "bf16" else 4
+
+
+# --------------------------------------------------------------------------------------------------
+# multi-rank plumbing (ranks are independent replicas; the only collective is the max over times)
+# --------------------------------------------------------------------------------------------------
+def dist_setup(n_gpus: int):
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist.init_process_group(backend=backend)
+        return dist.get_rank(), world, int(os.environ.get("LOCAL_RANK", "0"))
+    return 0, 1, 0
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(local_ms: float, world: int, device: str) -> float:
+    """Slowest rank's time: the step count is fixed per rank, so whole-job throughput divides by this."""
+    if world == 1:
+        return local_ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(device_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        rows = [r.strip().split(",") for r in self.tmp.read().splitlines() if r.strip()]
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                power.append(float(r[2]))
+                for name, v in zip(names, r[3:7]):
+                    if v.strip().lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       power_w_max=max(power))
+        return out
+
+
+# --------------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------------
+class Runner:
+    """Owns the buffers of one workload and runs steps through the C ABI."""
+
+    def __init__(self, w, device_index: int, n_batches: int = 2, rank: int = 0):
+        import torch
+        from paper_2507_05508_b200 import binding as B
+        from paper_2507_05508_b200 import workloads as wl
+        self.torch, self.B, self.wl, self.w = torch, B, wl, w
+        self.dev = f"cuda:{device_index}"
+        torch.cuda.set_device(device_index)
+        self.ctx = B.mlmc_create(device_index, w.d, w.M, 32)
+        sc = wl.scales(w, self.dev)
+        self.batches = [wl.gradients(w, 1000 * rank + i, self.dev, sc) for i in range(n_batches)]
+        del sc
+        self.dense = torch.empty(w.d, dtype=torch.float32, device=self.dev)
+        if w.kind == "topk":
+            self.k = wl.topk_schedule(w)
+            self.L = len(self.k)
+            self.msgs = B.TopkBuffers(w.M, wl.max_band(self.k), self.dev)
+        else:
+            self.b = list(w.bits)
+            self.L = len(self.b)
+            widths = [self.b[0]] + [self.b[i] - self.b[i - 1] for i in range(1, self.L)]
+            self.msgs = B.BitBuffers(w.M, w.d, max(widths), self.dev)
+        self.p = None if w.adaptive else list(wl.geometric_probs(self.L))
+        torch.cuda.synchronize()
+
+    def step(self, i: int, g=None):
+        B, w = self.B, self.w
+        g = self.batches[i % len(self.batches)] if g is None else g
+        if w.kind == "topk":
+            B.mlmc_compress_topk(self.ctx, g, self.k, self.p, w.seed, i, self.msgs)
+            B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, self.msgs, None, w.M, w.d, self.dense)
+        else:
+            B.mlmc_compress_bitwise(self.ctx, g, self.b, self.p, w.seed, i, self.msgs)
+            B.mlmc_aggregate(self.ctx, B.MLMC_BITWISE, self.msgs, self.b, w.M, w.d, self.dense)
+
+    def message_bytes(self) -> float:
+        """Bytes of the messages of the last step (written once by compress, read once by aggregate)."""
+        if self.w.kind == "topk":
+            return float(self.msgs.count.sum().item()) * 8.0
+        widths = [self.b[0]] + [self.b[i] - self.b[i - 1] for i in range(1, self.L)]
+        lv = self.msgs.level.tolist()
+        return float(sum((1 + widths[l]) * self.msgs.words * 4 for l in lv if l >= 0))
+
+    def close(self):
+        self.B.mlmc_destroy(self.ctx)
+
+
+def sweeps_charged(w) -> int:
+    """Gradient sweeps the method needs (a true data dependence separates them): select -> emit for Top-k,
+    max -> pack for fixed-p bit-wise, max -> field energies -> pack for adaptive bit-wise."""
+    if w.kind == "topk":
+        return 2
+    return 3 if w.adaptive else 2
+
+
+# Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes, dense bytes).
+def kernel_alg_bytes(name: str, sweep: float, msg: float, dense: float):
+    table = {
+        "hist1": sweep, "masked_pass2": sweep, "masked_pass3": sweep, "norm_sweep": sweep,
+        "emit": sweep + msg, "aggregate_topk": msg + dense,
+        "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + msg, "aggregate_bitwise": msg + dense,
+    }
+    return table.get(name)
+
+
+def run_cuda(args):
+    import torch
+    from paper_2507_05508_b200 import build as cuda_build
+    from paper_2507_05508_b200 import workloads as wl
+    cuda_build.build()
+    rank, world, local = dist_setup(args.gpus)
+    w = wl.ALL[args.workload]
+    peak, peak_kind = measured_peak()
+    r = Runner(w, local, rank=rank)
+    B = r.B
+    sweep_bytes = float(w.M) * w.d * elem_size(w)
+    dense_bytes = float(w.d) * 4.0
+
+    for i in range(max(args.warmup, 3)):
+        r.step(i)
+    torch.cuda.synchronize()
+    assert B.mlmc_get_status(r.ctx) == 0, "device status after warm-up"
+
+    # ---- timed region: exactly K steps, device-timed, per-kernel event pairs on the same stream
+    B.mlmc_timing_enable(r.ctx, True)
+    launches0 = B.mlmc_launch_count(r.ctx)
+    msg_bytes_total = 0.0
+    sampler = ClockSampler(local)
+    barrier(world)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        r.step(args.warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    t_wall = time.time() - t_wall0
+    clocks = sampler.stop()
+    local_ms = e0.elapsed_time(e1)
+    total_ms = max_over_ranks(local_ms, world, r.dev)
+    launches = B.mlmc_launch_count(r.ctx) - launches0
+    per_kernel = B.mlmc_timing_read(r.ctx)
+    B.mlmc_timing_enable(r.ctx, False)
+    status = B.mlmc_get_status(r.ctx)
+    ms_per_step = total_ms / args.steps
+    value = world * sweep_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # message volume: average over a few steps outside the timed region (levels are redrawn every step)
+    probe = min(args.steps, 8)
+    for i in range(probe):
+        r.step(args.warmup + i)
+        msg_bytes_total += r.message_bytes()
+    msg_bytes = msg_bytes_total / probe
+
+    # ---- roofline of the dominant kernel and of the whole step
+    dom = max(per_kernel.items(), key=lambda kv: kv[1][0])
+    dom_name, (dom_ms, dom_n) = dom
+    dom_bytes = kernel_alg_bytes(dom_name, sweep_bytes, msg_bytes, dense_bytes) or sweep_bytes
+    dom_avg_s = dom_ms / dom_n * 1e-3
+    achieved = dom_bytes / dom_avg_s / 1e9
+    ratio = NCU_TRAFFIC_RATIO.get(f"{dom_name}:{w.dtype}")
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "peak_source": peak_kind,
+                "traffic": None if ratio is None else ratio * dom_bytes,
+                "alg_bytes_per_launch": dom_bytes, "avg_launch_ms": round(dom_avg_s * 1e3, 4)}
+    b_alg = sweeps_charged(w) * sweep_bytes + 2 * msg_bytes + dense_bytes
+    step_frac = b_alg / (ms_per_step * 1e-3) / 1e9 / peak
+    kernels = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] / args.steps,
+                   "share": round(v[0] / sum(x[0] for x in per_kernel.values()), 4)}
+               for k, v in sorted(per_kernel.items(), key=lambda kv: -kv[1][0])}
+
+    # ---- end to end: inputs start in pinned host memory, the dense mean ends in host memory
+    e2e = None
+    if args.e2e_steps > 0:
+        host_in = torch.empty(r.batches[0].shape, dtype=r.batches[0].dtype, pin_memory=True)
+        host_in.copy_(r.batches[0])
+        host_out = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
+        g_dev = r.batches[1 % len(r.batches)]
+
+        def e2e_step(i):
+            g_dev.copy_(host_in, non_blocking=True)
+            r.step(i, g_dev)
+            host_out.copy_(r.dense, non_blocking=True)
+
+        e2e_step(0)
+        torch.cuda.synchronize()
+        barrier(world)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(args.e2e_steps):
+            e2e_step(i + 1)
+        b.record()
+        torch.cuda.synchronize()
+        barrier(world)
+        e2e_ms = max_over_ranks(a.elapsed_time(b), world, r.dev) / args.e2e_steps
+        e2e = {"value": round(world * sweep_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
+               "h2d_bytes_per_step": int(sweep_bytes), "d2h_bytes_per_step": int(dense_bytes),
+               "ms_per_step": round(e2e_ms, 3)}
+        del host_in, host_out
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(w, r.batches[0][0], budget_s=15.0)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}: {'adaptive' if w.adaptive else 'fixed-p'} MLMC-{w.kind}, d={w.d}, "
+                                   f"M={w.M}, {w.dtype}, L={r.L}", "l2_policy": "inputs larger than L2: "
+                       f"{sweep_bytes / 1e6:.0f} MB per sweep, 2 batches alternated", "parallelism": "replicas only"},
+            "elements_per_s": round(world * w.M * w.d / (ms_per_step * 1e-3), 1),
+            "step_roofline": {"alg_bytes_per_step": b_alg, "sweeps_charged": sweeps_charged(w),
+                              "message_bytes_per_step": msg_bytes, "frac_of_peak": round(step_frac, 4),
+                              "frac_of_8TBs": round(b_alg / (ms_per_step * 1e-3) / 8e12, 4)},
+            "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "e2e": e2e,
+            "cpu_baseline": cpu, "clocks": clocks, "device_status": status, "wall_s_timed": round(t_wall, 3),
+        }
+        print(json.dumps(line))
+    r.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------------
+# the oracle, timed on the host cores (reported baseline, and the --impl reference arm)
+# --------------------------------------------------------------------------------------------------
+def oracle_sample_step(w, g_row_np, d_s: int, step: int):
+    """One worker's compress + its aggregate share on the first d_s coordinates; returns seconds."""
+    import numpy as np
+    import oracle
+    from paper_2507_05508_b200 import workloads as wl
+    x = np.ascontiguousarray(g_row_np[:d_s])
+    t0 = time.perf_counter()
+    if w.kind == "topk":
+        ws = wl.shrink(w, d_s, 1)
+        k = wl.topk_schedule(ws)
+        p = None if w.adaptive else wl.geometric_probs(len(k))
+        m = oracle.topk(x, k, p=p, seed=w.seed, step=step, worker=0)
+        oracle.aggregate_topk([(m.idx, m.val)], d_s)
+    else:
+        b = list(w.bits)
+        p = None if w.adaptive else wl.geometric_probs(len(b))
+        m = oracle.bitwise(x, b, p=p, seed=w.seed, step=step, worker=0)
+        oracle.aggregate_bitwise([m], b, d_s)
+    return time.perf_counter() - t0
+
+
+def calibrate_sample(w, g_row_np, budget_s: float) -> int:
+    """Largest power-of-two prefix whose oracle step fits the per-step budget (extrapolated from a probe)."""
+    probe = min(1 << 18, w.d)
+    t = max(oracle_sample_step(w, g_row_np, probe, 0), 1e-4)
+    d_s = probe
+    while d_s * 2 <= min(w.d, 1 << 25) and t * 2.2 <= budget_s:
+        d_s *= 2
+        t *= 2.2
+    return d_s
+
+
+def cpu_baseline(w, g_row, budget_s: float):
+    import oracle
+    from paper_2507_05508_b200 import workloads as wl
+    oracle.build()
+    row = wl.as_numpy_bits(g_row.unsqueeze(0))[0]
+    d_s = calibrate_sample(w, row, budget_s)
+    t = oracle_sample_step(w, row, d_s, 1)
+    return {"value": round(d_s * elem_size(w) / t / 1e9, 5), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"1 worker, first {d_s} of d={w.d} coordinates, compress + aggregate, {t:.2f} s",
+            "elements_per_s": round(d_s / t, 1)}
+
+
+def run_reference(args):
+    """Times the CPU oracle, as it stands, on bounded samples of the same workload (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2507_05508_b200 import workloads as wl
+    oracle.build()
+    w = wl.ALL[args.workload]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    d_gen = min(w.d, 1 << 25)
+    wg = wl.shrink(w, d_gen, 1) if d_gen < w.d else w
+    row = wl.as_numpy_bits(wl.gradients(wg, 0, dev)[:1])[0]
+    per_step_budget = max(0.05, 150.0 / max(1, args.steps + args.warmup))
+    d_s = min(calibrate_sample(w, row, per_step_budget), d_gen)
+    for i in range(args.warmup):
+        oracle_sample_step(w, row, d_s, i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle_sample_step(w, row, d_s, args.warmup + i)
+    t = (time.perf_counter() - t0) / args.steps
+    value = d_s * elem_size(w) / t / 1e9
+    sample = f"each step: 1 worker, first {d_s} of d={w.d} coordinates, compress + aggregate on 1 host core"
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(t * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.dtype == "f32" else "bf16", "data": "synthetic",
+            "config": {"workload": f"{w.name}: {'adaptive' if w.adaptive else 'fixed-p'} MLMC-{w.kind}, d={w.d}, "
+                                   f"M={w.M}, {w.dtype}", "sample": sample},
+            "cpu_baseline": {"value": round(value, 5), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 5), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_cuda(a)

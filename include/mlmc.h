@@ -91,6 +91,16 @@ int mlmc_get_status(mlmc_ctx* ctx, void* stream);
 /* Number of kernels this ctx has launched so far (host counter; for launch accounting). */
 int64_t mlmc_launch_count(const mlmc_ctx* ctx);
 
+/* Per-kernel timing for roofline measurements (instrumentation of this library; not part of the
+ * method).  With timing on, every kernel launch is bracketed by a CUDA event pair on its stream (at
+ * most 2048 launches between two reads; later ones are not recorded).  mlmc_timing_read synchronises
+ * `stream`, fills total_ms[id] and launches[id] for id < mlmc_kernel_count() (host arrays) with the
+ * launches recorded since the previous read, and restarts the record. */
+int mlmc_kernel_count(void);
+const char* mlmc_kernel_name(int id);
+int mlmc_timing_enable(mlmc_ctx* ctx, int on);
+int mlmc_timing_read(mlmc_ctx* ctx, double* total_ms, int64_t* launches, void* stream);
+
 /* The uniforms of the level draw for workers 0..M-1 at (seed, step), computed on the device and
  * copied to u_host[M].  Synchronous; for checking the counter generator against known answers. */
 int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream);

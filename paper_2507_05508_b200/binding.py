@@ -23,6 +23,7 @@ MLMC_ERR_NONFINITE, MLMC_ERR_TIMEOUT, MLMC_ERR_CUDA, MLMC_ERR_NOMEM, MLMC_ERR_IN
 MLMC_MAX_LEVELS = 32
 
 EXPORTS = ["mlmc_create", "mlmc_destroy", "mlmc_get_status", "mlmc_launch_count", "mlmc_read_u",
+           "mlmc_kernel_count", "mlmc_kernel_name", "mlmc_timing_enable", "mlmc_timing_read",
            "mlmc_level_probs", "mlmc_compress_topk", "mlmc_compress_bitwise", "mlmc_aggregate"]
 
 
@@ -64,9 +65,14 @@ def lib() -> C.CDLL:
         L.mlmc_compress_topk.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_compress_bitwise.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_aggregate.argtypes = [vp, i32, vp, vp, i32, i32, i64, vp, vp]
+        L.mlmc_kernel_count.argtypes = []
+        L.mlmc_kernel_name.argtypes = [i32]
+        L.mlmc_timing_enable.argtypes = [vp, i32]
+        L.mlmc_timing_read.argtypes = [vp, vp, vp, vp]
         for name in EXPORTS:
-            if name != "mlmc_launch_count":
+            if name not in ("mlmc_launch_count", "mlmc_kernel_name"):
                 getattr(L, name).restype = i32
+        L.mlmc_kernel_name.restype = C.c_char_p
         _lib = L
     return _lib
 
@@ -110,6 +116,26 @@ def mlmc_get_status(ctx) -> int:
 
 def mlmc_launch_count(ctx) -> int:
     return int(lib().mlmc_launch_count(ctx))
+
+
+def mlmc_kernel_count() -> int:
+    return int(lib().mlmc_kernel_count())
+
+
+def mlmc_kernel_name(i: int) -> str:
+    return lib().mlmc_kernel_name(i).decode()
+
+
+def mlmc_timing_enable(ctx, on: bool) -> None:
+    _check(lib().mlmc_timing_enable(ctx, 1 if on else 0), "mlmc_timing_enable")
+
+
+def mlmc_timing_read(ctx):
+    """{kernel name: (total ms, launches)} recorded since the previous read (synchronises the stream)."""
+    n = mlmc_kernel_count()
+    ms, cnt = (C.c_double * n)(), (C.c_int64 * n)()
+    _check(lib().mlmc_timing_read(ctx, ms, cnt, _stream()), "mlmc_timing_read")
+    return {mlmc_kernel_name(i): (ms[i], cnt[i]) for i in range(n) if cnt[i]}
 
 
 def mlmc_read_u(ctx, seed: int, step: int, M: int):

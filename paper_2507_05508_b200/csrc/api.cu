@@ -126,6 +126,11 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.L_max = L_max;
     ws.sm_count = prop.multiProcessorCount;
     ws.launches = 0;
+    ws.timing = false;
+    ws.timing_used = 0;
+    ws.ev_start = ws.ev_stop = nullptr;
+    ws.ev_id = nullptr;
+    for (int i = 0; i < K_COUNT; ++i) ws.launches_by_id[i] = 0;
     ws.norm_ctas = ws.sm_count * 4;
     ws.stat_ctas = ws.sm_count * 4;
     const int64_t emit_tiles = (d_max + kEmitTile - 1) / kEmitTile;
@@ -203,6 +208,15 @@ int mlmc_destroy(mlmc_ctx* ctx) {
     if (!ctx) return MLMC_ERR_ARG;
     DeviceGuard guard(ctx->ws.device);
     cudaDeviceSynchronize();
+    if (ctx->ws.ev_start) {
+        for (int i = 0; i < kTimingPool; ++i) {
+            cudaEventDestroy(ctx->ws.ev_start[i]);
+            cudaEventDestroy(ctx->ws.ev_stop[i]);
+        }
+        delete[] ctx->ws.ev_start;
+        delete[] ctx->ws.ev_stop;
+        delete[] ctx->ws.ev_id;
+    }
     const cudaError_t e = cudaFree(ctx->slab);
     delete ctx;
     return finish(e);
@@ -223,6 +237,52 @@ int mlmc_get_status(mlmc_ctx* ctx, void* stream) {
 }
 
 int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches : 0; }
+
+static const char* const kKernelNames[K_COUNT] = {
+    "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "masked_pass2", "resolve2", "masked_pass3",
+    "resolve3", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
+    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise"};
+
+int mlmc_kernel_count(void) { return K_COUNT; }
+
+const char* mlmc_kernel_name(int id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : ""; }
+
+int mlmc_timing_enable(mlmc_ctx* ctx, int on) {
+    if (!ctx) return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    DeviceGuard guard(ws.device);
+    if (on && !ws.ev_start) {
+        ws.ev_start = new (std::nothrow) cudaEvent_t[kTimingPool];
+        ws.ev_stop = new (std::nothrow) cudaEvent_t[kTimingPool];
+        ws.ev_id = new (std::nothrow) int[kTimingPool];
+        if (!ws.ev_start || !ws.ev_stop || !ws.ev_id) return MLMC_ERR_NOMEM;
+        for (int i = 0; i < kTimingPool; ++i)
+            if (cudaEventCreate(&ws.ev_start[i]) != cudaSuccess || cudaEventCreate(&ws.ev_stop[i]) != cudaSuccess)
+                return MLMC_ERR_CUDA;
+    }
+    ws.timing = on != 0;
+    ws.timing_used = 0;
+    return MLMC_OK;
+}
+
+int mlmc_timing_read(mlmc_ctx* ctx, double* total_ms, int64_t* launches, void* stream) {
+    if (!ctx || !total_ms || !launches) return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    DeviceGuard guard(ws.device);
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return MLMC_ERR_CUDA;
+    for (int i = 0; i < K_COUNT; ++i) {
+        total_ms[i] = 0.0;
+        launches[i] = 0;
+    }
+    for (int i = 0; i < ws.timing_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ws.ev_start[i], ws.ev_stop[i]) != cudaSuccess) return MLMC_ERR_CUDA;
+        total_ms[ws.ev_id[i]] += ms;
+        launches[ws.ev_id[i]]++;
+    }
+    ws.timing_used = 0;
+    return MLMC_OK;
+}
 
 int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream) {
     if (!ctx || !u_host || M < 1 || M > ctx->ws.M_max) return MLMC_ERR_ARG;

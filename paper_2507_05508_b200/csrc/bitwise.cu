@@ -309,6 +309,7 @@ int bit_blocks(const Workspace& ws, int64_t d, int vec, int M, int waves) {
 
 void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
     cudaMemsetAsync(ws.gmax_bits, 0, (size_t)M * sizeof(uint32_t), s);
+    LaunchScope t(ws, K_ABSMAX, s);
     if (dtype == MLMC_BF16) {
         const int nb = bit_blocks(ws, d, 8, M, 8);
         absmax_kernel<bf16_t><<<dim3(nb, M), kSweepThreads, 0, s>>>(static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits,
@@ -318,7 +319,6 @@ void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, in
         absmax_kernel<float><<<dim3(nb, M), kSweepThreads, 0, s>>>(static_cast<const float*>(g), d, ld, ws.gmax_bits,
                                                                    ws.status, ws.worker_err);
     }
-    ws.launches++;
 }
 
 template <typename T>
@@ -342,22 +342,22 @@ void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M,
     cudaMemsetAsync(ws.S_partial, 0, (size_t)M * ws.stat_ctas * kMaxLevels * sizeof(unsigned long long), s);
     int nb = bit_blocks(ws, d, dtype == MLMC_BF16 ? 8 : 4, M, 4);
     if (nb > ws.stat_ctas) nb = ws.stat_ctas;
+    LaunchScope t(ws, K_BIT_STATS, s);
     if (dtype == MLMC_BF16)
         launch_bit_stats_t<bf16_t>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, nb, s);
     else
         launch_bit_stats_t<float>(ws, static_cast<const float*>(g), d, M, ld, sc, nb, s);
-    ws.launches++;
 }
 
 void launch_bit_probs_draw(Workspace& ws, int M, const int32_t* b, int L, bool adaptive, bool need_delta,
                            uint64_t seed, uint64_t step, const mlmc_bit_msgs* out, cudaStream_t s) {
     const BitSchedule sc = make_schedule(b, L);
+    LaunchScope t(ws, K_BIT_DRAW, s);
     bit_probs_draw_kernel<<<(M + 63) / 64, 64, 0, s>>>(
         sc, ws.gmax_bits, ws.S_partial, ws.stat_ctas, ws.stat_ctas, ws.p_fixed, adaptive ? 1 : 0, need_delta ? 1 : 0,
         seed, step, M, ws.p_all, ws.delta_all, ws.u_dev, ws.bit_level, out ? out->gmax : nullptr,
         out ? out->level : nullptr, out ? out->p_sel : nullptr, out ? out->w_max : 0, out ? 1 : 0, ws.status,
         ws.worker_err);
-    ws.launches++;
 }
 
 void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
@@ -369,13 +369,13 @@ void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, 
     const int64_t cap = ((int64_t)ws.sm_count * 16 + M - 1) / M;
     if (nb > cap) nb = cap;
     if (nb < 1) nb = 1;
+    LaunchScope t(ws, K_BIT_PACK, s);
     if (dtype == MLMC_BF16)
         bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, 0, s>>>(
             static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
     else
         bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, 0, s>>>(
             static_cast<const float*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
-    ws.launches++;
 }
 
 void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const int32_t* b, int L, int M, int64_t d,
@@ -385,9 +385,9 @@ void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const in
     int64_t nb = (words + kBitThreads - 1) / kBitThreads;
     const int64_t cap = (int64_t)ws.sm_count * 8;
     if (nb > cap) nb = cap;
+    LaunchScope t(ws, K_AGG_BIT, s);
     aggregate_bitwise_kernel<<<(unsigned)nb, kBitThreads, 0, s>>>(msgs.planes, msgs.gmax, msgs.level, msgs.p_sel, sc,
                                                                   msgs.w_max, words, M, d, out);
-    ws.launches++;
 }
 
 }  // namespace mlmc

@@ -52,7 +52,23 @@ struct TileRec {
     uint32_t flag;
 };
 
+// Kernel identifiers for launch accounting and per-kernel timing.
+enum KernelId {
+    K_DRAW_FIXED = 0, K_INIT_QUERIES, K_UNIFORMS, K_HIST1, K_RESOLVE1, K_MASKED2, K_RESOLVE2, K_MASKED3, K_RESOLVE3,
+    K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
+    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_COUNT
+};
+
+constexpr int kTimingPool = 2048;  // event pairs kept between two reads
+
 struct Workspace {
+    // per-kernel timing (off by default): one CUDA event pair around every kernel launch
+    bool timing;
+    int timing_used;
+    cudaEvent_t* ev_start;
+    cudaEvent_t* ev_stop;
+    int* ev_id;
+    int64_t launches_by_id[K_COUNT];
     int device;
     int64_t d_max;
     int M_max, L_max;
@@ -175,6 +191,25 @@ __device__ __forceinline__ void block_vector_range(int64_t d, int vec, int bx, i
     *v0 = min((int64_t)bx * per, nvec);
     *v1 = min(*v0 + per, nvec);
 }
+
+// Brackets one kernel launch: counts it and, when timing is on, records an event pair on the stream.
+struct LaunchScope {
+    Workspace& ws;
+    cudaStream_t s;
+    int slot;
+    LaunchScope(Workspace& w, int id, cudaStream_t st) : ws(w), s(st), slot(-1) {
+        ws.launches++;
+        ws.launches_by_id[id]++;
+        if (ws.timing && ws.timing_used < kTimingPool) {
+            slot = ws.timing_used++;
+            ws.ev_id[slot] = id;
+            cudaEventRecord(ws.ev_start[slot], s);
+        }
+    }
+    ~LaunchScope() {
+        if (slot >= 0) cudaEventRecord(ws.ev_stop[slot], s);
+    }
+};
 
 // ---------------------------------------------------------------------------------------------
 // launchers (each enqueues on `s` and bumps ws.launches)

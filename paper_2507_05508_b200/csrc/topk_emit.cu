@@ -277,6 +277,7 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
     cudaMemsetAsync(ws.tile_counter, 0, sizeof(unsigned), s);
     unsigned grid = (unsigned)ws.sm_count * 8u;
     if (grid > total) grid = total;
+    LaunchScope t(ws, K_EMIT, s);
     if (dtype == MLMC_BF16)
         emit_kernel<bf16_t><<<grid, kEmitThreads, 0, s>>>(static_cast<const bf16_t*>(g), d, ld, tpw, total, ws.emit,
                                                          ws.tile_agg, ws.tile_inc, ws.tile_counter, out.idx, out.val,
@@ -285,19 +286,20 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
         emit_kernel<float><<<grid, kEmitThreads, 0, s>>>(static_cast<const float*>(g), d, ld, tpw, total, ws.emit,
                                                         ws.tile_agg, ws.tile_inc, ws.tile_counter, out.idx, out.val,
                                                         out.capacity, ws.status, ws.worker_err);
-    ws.launches++;
 }
 
 void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int64_t d, float* out, cudaStream_t s) {
     const int ntiles = (int)((d + kAggTile - 1) / kAggTile);
     const int64_t n_off = (int64_t)M * (ntiles + 1);
-    agg_offsets_kernel<<<(unsigned)((n_off + 255) / 256), 256, 0, s>>>(msgs.idx, msgs.count, msgs.level, msgs.capacity,
-                                                                       M, ntiles, ws.agg_offsets);
-    ws.launches++;
+    {
+        LaunchScope t(ws, K_AGG_OFFSETS, s);
+        agg_offsets_kernel<<<(unsigned)((n_off + 255) / 256), 256, 0, s>>>(msgs.idx, msgs.count, msgs.level,
+                                                                           msgs.capacity, M, ntiles, ws.agg_offsets);
+    }
     int grid = ws.sm_count * 8;
     if (grid > ntiles) grid = ntiles;
+    LaunchScope t(ws, K_AGG_TOPK, s);
     aggregate_topk_kernel<<<grid, 256, 0, s>>>(msgs.idx, msgs.val, msgs.capacity, M, d, ntiles, ws.agg_offsets, out);
-    ws.launches++;
 }
 
 }  // namespace mlmc

@@ -538,28 +538,31 @@ int blocks_per_worker(const Workspace& ws, int64_t d, int vec, int threads, int 
 // ---------------------------------------------------------------------------------------------
 void launch_init_queries_adaptive(Workspace& ws, int M, int L, int64_t d, cudaStream_t s) {
     if (L > 1) {
+        LaunchScope t(ws, K_INIT_QUERIES, s);
         init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 0);
-        ws.launches++;
     }
 }
 
 void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, cudaStream_t s) {
-    draw_fixed_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.p_fixed, L, seed, step, ws.p_all, ws.u_dev, ws.emit, M);
-    ws.launches++;
+    {
+        LaunchScope t(ws, K_DRAW_FIXED, s);
+        draw_fixed_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.p_fixed, L, seed, step, ws.p_all, ws.u_dev, ws.emit, M);
+    }
     if (L > 1) {
+        LaunchScope t(ws, K_INIT_QUERIES, s);
         init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 1);
-        ws.launches++;
     }
 }
 
 void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStream_t s) {
+    LaunchScope t(ws, K_UNIFORMS, s);
     uniforms_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.u_dev, M, seed, step);
-    ws.launches++;
 }
 
 void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
     cudaMemsetAsync(ws.hist1, 0, (size_t)M * kBins1 * sizeof(uint32_t), s);
     const size_t smem = kBins1 * sizeof(uint32_t);
+    LaunchScope t(ws, K_HIST1, s);
     if (dtype == MLMC_BF16) {
         const int nb = blocks_per_worker(ws, d, 8, kHistThreads, M, 2);
         hist1_kernel<bf16_t><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const bf16_t*>(g), d, ld, ws.hist1,
@@ -569,14 +572,13 @@ void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int
         hist1_kernel<float><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.hist1,
                                                                     ws.status, ws.worker_err);
     }
-    ws.launches++;
 }
 
 void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
     if (dtype != MLMC_BF16) cudaMemsetAsync(ws.table1, 0xFF, (size_t)M * kBins1, s);
+    LaunchScope t(ws, K_RESOLVE1, s);
     resolve1_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, ws.table1, L - 1, dtype == MLMC_BF16,
                                                   ws.worker_err);
-    ws.launches++;
 }
 
 void launch_masked_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s) {
@@ -586,22 +588,23 @@ void launch_masked_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t 
     if (pass == 2) {
         cudaMemsetAsync(ws.hist2, 0, hist_bytes, s);
         cudaMemsetAsync(ws.map2, 0xFF, (size_t)M * kMaxQueries * kBins23, s);
+        LaunchScope t(ws, K_MASKED2, s);
         masked_pass_kernel<2><<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.table1,
                                                                        ws.map2, ws.hist2, ws.worker_err);
     } else {
         cudaMemsetAsync(ws.hist3, 0, hist_bytes, s);
+        LaunchScope t(ws, K_MASKED3, s);
         masked_pass_kernel<3><<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.table1,
                                                                        ws.map2, ws.hist3, ws.worker_err);
     }
-    ws.launches++;
 }
 
 void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
+    LaunchScope t(ws, pass == 2 ? K_RESOLVE2 : K_RESOLVE3, s);
     if (pass == 2)
         resolve23_kernel<2><<<M, kResolveThreads, 0, s>>>(ws.hist2, ws.queries, ws.map2, L - 1, ws.worker_err);
     else
         resolve23_kernel<3><<<M, kResolveThreads, 0, s>>>(ws.hist3, ws.queries, ws.map2, L - 1, ws.worker_err);
-    ws.launches++;
 }
 
 void launch_norm_sweep(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
@@ -609,32 +612,32 @@ void launch_norm_sweep(Workspace& ws, const void* g, int64_t d, int M, int64_t l
     if (nb > ws.norm_ctas) nb = ws.norm_ctas;
     const size_t smem = (size_t)L * kSweepThreads * sizeof(double);
     cudaMemsetAsync(ws.band_partial, 0, (size_t)M * ws.norm_ctas * kMaxLevels * sizeof(double), s);
+    LaunchScope t(ws, K_NORM_SWEEP, s);
     norm_sweep_kernel<<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.queries, L,
                                                                ws.band_partial, ws.norm_ctas, ws.worker_err);
-    ws.launches++;
 }
 
 void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s) {
+    LaunchScope t(ws, K_NORM_HIST, s);
     norm_from_hist_bf16_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, L, ws.band_partial, ws.norm_ctas,
                                                              ws.worker_err);
-    ws.launches++;
 }
 
 void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool adaptive, bool want_emit,
                        uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, cudaStream_t s) {
     const int n_partials = (dtype == MLMC_BF16) ? 1 : ws.norm_ctas;
+    LaunchScope t(ws, K_PROBS_DRAW, s);
     probs_draw_kernel<<<M, kMaxLevels, 0, s>>>(
         ws.queries, ws.k_dev, L, d, dtype == MLMC_BF16, ws.band_partial, n_partials, ws.norm_ctas, adaptive ? 1 : 0,
         seed, step, ws.p_all, ws.delta_all, ws.u_dev, ws.emit, out ? out->count : nullptr, out ? out->level : nullptr,
         out ? out->p_sel : nullptr, out ? out->capacity : 0, ws.status, ws.worker_err, want_emit ? 1 : 0);
-    ws.launches++;
 }
 
 void launch_copy_probs(Workspace& ws, int M, int L, const double* p_fixed, double* p_out, double* delta_out,
                        cudaStream_t s) {
+    LaunchScope t(ws, K_COPY_PROBS, s);
     copy_probs_kernel<<<(M * L + 127) / 128, 128, 0, s>>>(ws.p_all, ws.delta_all, p_fixed, M, L, p_out, delta_out,
                                                           ws.worker_err);
-    ws.launches++;
 }
 
 int configure_select_kernels() {
