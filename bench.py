@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shrink-d", type=int, default=0, help="profiling aid: same workload structure at a smaller d")
+    ap.add_argument("--shrink-M", type=int, default=0)
     return ap.parse_args()
 
 
@@ -202,7 +204,7 @@ def sweeps_charged(w) -> int:
 # Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes, dense bytes).
 def kernel_alg_bytes(name: str, sweep: float, msg: float, dense: float):
     table = {
-        "hist1": sweep, "masked_pass2": sweep, "masked_pass3": sweep, "norm_sweep": sweep,
+        "hist1": sweep, "sums_candidates": sweep, "masked_pass2": sweep, "masked_pass3": sweep, "norm_sweep": sweep,
         "emit": sweep + msg, "aggregate_topk": msg + dense,
         "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + msg, "aggregate_bitwise": msg + dense,
     }
@@ -216,6 +218,8 @@ def run_cuda(args):
     cuda_build.build()
     rank, world, local = dist_setup(args.gpus)
     w = wl.ALL[args.workload]
+    if args.shrink_d or args.shrink_M:
+        w = wl.shrink(w, args.shrink_d or w.d, args.shrink_M or w.M)
     peak, peak_kind = measured_peak()
     r = Runner(w, local, rank=rank)
     B = r.B

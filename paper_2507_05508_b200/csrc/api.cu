@@ -86,14 +86,20 @@ int normalise_probs(const double* p, int L, double* out) {
 int finish(cudaError_t e) { return e == cudaSuccess ? MLMC_OK : MLMC_ERR_CUDA; }
 
 // Thresholds of every live query (sweep 1 + the two masked digit passes for fp32).
-void run_selection(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
+// sweep 1 (leading-digit histogram), and for fp32 sweep 2 (candidates [+ energies]) and the two remaining
+// digit passes over the candidates.
+void run_selection(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, int L, bool sums,
+                   cudaStream_t s) {
     launch_hist1(ws, g, dtype, d, M, ld, s);
     launch_resolve1(ws, dtype, M, L, s);
-    if (dtype == MLMC_F32 && L > 1) {
-        launch_masked_pass(ws, g, d, M, ld, 2, s);
-        launch_resolve23(ws, M, L, 2, s);
-        launch_masked_pass(ws, g, d, M, ld, 3, s);
-        launch_resolve23(ws, M, L, 3, s);
+    if (dtype == MLMC_F32) {
+        launch_sums_candidates(ws, g, d, M, ld, L, sums, s);
+        if (L > 1) {
+            launch_digit_pass(ws, g, d, M, ld, 2, s);
+            launch_resolve23(ws, M, L, 2, s);
+            launch_digit_pass(ws, g, d, M, ld, 3, s);
+            launch_resolve23(ws, M, L, 3, s);
+        }
     }
 }
 
@@ -101,7 +107,7 @@ void run_band_norms(Workspace& ws, const void* g, int dtype, int64_t d, int M, i
     if (dtype == MLMC_BF16)
         launch_norm_from_hist_bf16(ws, M, L, s);
     else
-        launch_norm_sweep(ws, g, d, M, ld, L, s);
+        launch_band_norms_fp32(ws, g, d, M, ld, L, s);
 }
 
 }  // namespace
@@ -132,6 +138,11 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.ev_id = nullptr;
     for (int i = 0; i < K_COUNT; ++i) ws.launches_by_id[i] = 0;
     ws.norm_ctas = ws.sm_count * 4;
+    ws.sum_ctas = ws.sm_count * 4;
+    ws.cand_ctas = ws.sm_count * 2;
+    ws.cur_norm_ctas = ws.cur_sum_ctas = ws.cur_cand_ctas = 0;
+    // candidate keys: a quarter of the row (boundary bins normally hold a few percent of it); small rows fit whole
+    ws.cand_cap = d_max / 4 > (int64_t(1) << 20) ? d_max / 4 : (d_max < (int64_t(1) << 20) ? d_max : (int64_t(1) << 20));
     ws.stat_ctas = ws.sm_count * 4;
     const int64_t emit_tiles = (d_max + kEmitTile - 1) / kEmitTile;
     const int64_t agg_tiles = (d_max + kAggTile - 1) / kAggTile;
@@ -147,15 +158,19 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_hist3 = pl.take(sizeof(uint32_t) * kMaxQueries * kBins23 * M_max);
     const size_t o_queries = pl.take(sizeof(Query) * kMaxQueries * M_max);
     const size_t o_band = pl.take(sizeof(double) * kMaxLevels * ws.norm_ctas * M_max);
+    const size_t o_sum = pl.take(sizeof(double) * kMaxLevels * ws.sum_ctas * M_max);
+    const size_t o_cpart = pl.take(sizeof(double) * kMaxLevels * ws.cand_ctas * M_max);
+    const size_t o_ckeys = pl.take(sizeof(uint32_t) * ws.cand_cap * M_max);
+    const size_t o_ccount = pl.take(sizeof(uint32_t) * M_max);
+    const size_t o_cover = pl.take(sizeof(int) * M_max);
     const size_t o_k = pl.take(sizeof(int64_t) * kMaxLevels);
     const size_t o_pfix = pl.take(sizeof(double) * kMaxLevels);
     const size_t o_pall = pl.take(sizeof(double) * kMaxLevels * M_max);
     const size_t o_dall = pl.take(sizeof(double) * kMaxLevels * M_max);
     const size_t o_u = pl.take(sizeof(double) * M_max);
     const size_t o_emit = pl.take(sizeof(EmitParams) * M_max);
-    const size_t o_tagg = pl.take(sizeof(TileRec) * ws.max_tiles);
-    const size_t o_tinc = pl.take(sizeof(TileRec) * ws.max_tiles);
-    const size_t o_tcnt = pl.take(sizeof(unsigned));
+    const size_t o_tdesc = pl.take(sizeof(uint4) * ws.max_tiles);
+    const size_t o_tcnt = pl.take(sizeof(unsigned) * M_max);
     const size_t o_aggoff = pl.take(sizeof(uint32_t) * (agg_tiles + 1) * M_max);
     const size_t o_gmax = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_S = pl.take(sizeof(unsigned long long) * kMaxLevels * ws.stat_ctas * M_max);
@@ -182,14 +197,18 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.hist3 = reinterpret_cast<uint32_t*>(base + o_hist3);
     ws.queries = reinterpret_cast<Query*>(base + o_queries);
     ws.band_partial = reinterpret_cast<double*>(base + o_band);
+    ws.sum_partial = reinterpret_cast<double*>(base + o_sum);
+    ws.cand_partial = reinterpret_cast<double*>(base + o_cpart);
+    ws.cand_keys = reinterpret_cast<uint32_t*>(base + o_ckeys);
+    ws.cand_count = reinterpret_cast<uint32_t*>(base + o_ccount);
+    ws.cand_overflow = reinterpret_cast<int*>(base + o_cover);
     ws.k_dev = reinterpret_cast<int64_t*>(base + o_k);
     ws.p_fixed = reinterpret_cast<double*>(base + o_pfix);
     ws.p_all = reinterpret_cast<double*>(base + o_pall);
     ws.delta_all = reinterpret_cast<double*>(base + o_dall);
     ws.u_dev = reinterpret_cast<double*>(base + o_u);
     ws.emit = reinterpret_cast<EmitParams*>(base + o_emit);
-    ws.tile_agg = reinterpret_cast<TileRec*>(base + o_tagg);
-    ws.tile_inc = reinterpret_cast<TileRec*>(base + o_tinc);
+    ws.tile_desc = reinterpret_cast<uint4*>(base + o_tdesc);
     ws.tile_counter = reinterpret_cast<unsigned*>(base + o_tcnt);
     ws.agg_offsets = reinterpret_cast<uint32_t*>(base + o_aggoff);
     ws.gmax_bits = reinterpret_cast<uint32_t*>(base + o_gmax);
@@ -239,8 +258,8 @@ int mlmc_get_status(mlmc_ctx* ctx, void* stream) {
 int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches : 0; }
 
 static const char* const kKernelNames[K_COUNT] = {
-    "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "masked_pass2", "resolve2", "masked_pass3",
-    "resolve3", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
+    "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "sums_candidates", "cand_pass2", "masked_pass2",
+    "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
     "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
@@ -318,7 +337,7 @@ int mlmc_level_probs(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, 
         cudaMemcpyAsync(ws.k_dev, sched, sizeof(int64_t) * L, cudaMemcpyHostToDevice, s);
         if (need_data) {
             launch_init_queries_adaptive(ws, M, L, d, s);
-            run_selection(ws, g, dtype, d, M, ld, L, s);
+            run_selection(ws, g, dtype, d, M, ld, L, true, s);
             run_band_norms(ws, g, dtype, d, M, ld, L, s);
             launch_probs_draw(ws, dtype, M, L, d, true, false, 0, 0, nullptr, s);
         }
@@ -355,7 +374,7 @@ int mlmc_compress_topk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M
         cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
         launch_draw_fixed(ws, M, L, d, seed, step, s);  // the draw does not depend on the data: only two thresholds are needed
     }
-    run_selection(ws, g, dtype, d, M, ld, L, s);
+    run_selection(ws, g, dtype, d, M, ld, L, adaptive, s);
     if (adaptive) run_band_norms(ws, g, dtype, d, M, ld, L, s);
     launch_probs_draw(ws, dtype, M, L, d, adaptive, true, seed, step, out, s);
     launch_emit(ws, g, dtype, d, M, ld, *out, s);

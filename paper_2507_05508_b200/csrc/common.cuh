@@ -16,7 +16,7 @@ constexpr uint32_t kKeyNone = 0xFFFFFFFFu;    // threshold above every finite ke
 constexpr uint32_t kNoSlot = 0xFFu;
 
 constexpr int kSweepThreads = 512;            // histogram / masked / norm sweeps
-constexpr int kEmitThreads = 256;
+constexpr int kEmitThreads = 128;
 constexpr int kEmitItems = 16;                // elements per thread per tile
 constexpr int kEmitTile = kEmitThreads * kEmitItems;
 constexpr int kAggTile = 4096;                // dense output elements per aggregation tile
@@ -46,16 +46,10 @@ struct EmitParams {
     int32_t pad;
 };
 
-// Look-back record of one emit tile: three running counts published once each.
-struct TileRec {
-    uint32_t D, Ea, Eb;
-    uint32_t flag;
-};
-
 // Kernel identifiers for launch accounting and per-kernel timing.
 enum KernelId {
-    K_DRAW_FIXED = 0, K_INIT_QUERIES, K_UNIFORMS, K_HIST1, K_RESOLVE1, K_MASKED2, K_RESOLVE2, K_MASKED3, K_RESOLVE3,
-    K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
+    K_DRAW_FIXED = 0, K_INIT_QUERIES, K_UNIFORMS, K_HIST1, K_RESOLVE1, K_SUMS_CAND, K_CAND2, K_MASKED2, K_RESOLVE2, K_CAND3,
+    K_MASKED3, K_RESOLVE3, K_CAND_SUMS, K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
     K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_COUNT
 };
 
@@ -83,18 +77,25 @@ struct Workspace {
     uint8_t* map2;               // [M][kMaxQueries][256] (slot2, digit2) -> slot of pass 3
     uint32_t* hist3;             // [M][kMaxQueries][256]
     Query* queries;              // [M][kMaxQueries]
-    double* band_partial;        // [M][norm_ctas][kMaxLevels] per-block open-interval sums
-    int norm_ctas;
+    double* band_partial;        // [M][norm_ctas][kMaxLevels] per-block open-interval sums (full sweep / bf16)
+    int norm_ctas, cur_norm_ctas;
+    double* sum_partial;         // [M][sum_ctas][kMaxLevels]  sweep 2: energy of the threshold-free bins
+    int sum_ctas, cur_sum_ctas;
+    double* cand_partial;        // [M][cand_ctas][kMaxLevels] energy of the candidate keys
+    int cand_ctas, cur_cand_ctas;
+    uint32_t* cand_keys;         // [M][cand_cap] keys of the boundary-bin elements
+    int64_t cand_cap;
+    uint32_t* cand_count;        // [M]
+    int* cand_overflow;          // [M] 1: the candidates did not fit, full-sweep passes take over
     int64_t* k_dev;              // [kMaxLevels] schedule
     double* p_fixed;             // [kMaxLevels] normalised fixed p
     double* p_all;               // [M][kMaxLevels]
     double* delta_all;           // [M][kMaxLevels]
     double* u_dev;               // [M]
     EmitParams* emit;            // [M]
-    TileRec* tile_agg;           // [max_tiles]
-    TileRec* tile_inc;           // [max_tiles]
+    uint4* tile_desc;            // [max_tiles] look-back records {D, Ea, Eb, state}
     int64_t max_tiles;
-    unsigned int* tile_counter;  // dynamic tile ticket
+    unsigned int* tile_counter;  // [M] ticket counters: tiles are numbered in the order they start
     uint32_t* agg_offsets;       // [M][agg_tiles_max + 1]
     // bit-wise
     uint32_t* gmax_bits;         // [M]
@@ -221,9 +222,11 @@ void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, ui
 void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStream_t s);
 void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s);
 void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s);
-void launch_masked_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s);
+void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,
+                            cudaStream_t s);
+void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s);
 void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s);
-void launch_norm_sweep(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s);
+void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s);
 void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s);
 void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool adaptive, bool want_emit,
                        uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, cudaStream_t s);

@@ -166,9 +166,13 @@ __device__ void assign_slots(Query* q, int nq, int shift) {
 
 // After sweep 1: suffix sums of the leading-digit histogram in place (S[b] = #{digit >= b}), then
 // every live query descends into its bin.  For bf16 the digit is the whole key, so the query is resolved.
+// For fp32 the kernel also writes the bin table of the second sweep: a bin that holds no threshold maps
+// to its open interval  #{ j : bin_j > b }  (code < 64); a bin that holds one maps to 64 + its slot.
 __global__ void __launch_bounds__(kResolveThreads, 1)
 resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is_bf16, const int* worker_err) {
     __shared__ uint32_t sh_warp[32];
+    __shared__ int sh_bin[kMaxQueries];
+    __shared__ uint32_t sh_slot[kMaxQueries];
     const int m = blockIdx.x;
     uint32_t* S = hist1 + (int64_t)m * kBins1;
     Query* q = queries + m * kMaxQueries;
@@ -202,26 +206,222 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is
         }
     }
     __syncthreads();
-    if (!is_bf16 && threadIdx.x == 0) {
-        assign_slots(q, nq, 16);
-        for (int j = 0; j < nq; ++j)
-            if (!q[j].trivial) table1[(int64_t)m * kBins1 + (q[j].prefix >> 16)] = (uint8_t)q[j].slot;
+    if (is_bf16) return;
+    if (threadIdx.x == 0) assign_slots(q, nq, 16);
+    __syncthreads();
+    if (threadIdx.x < nq) {
+        const Query& qq = q[threadIdx.x];
+        // trivial queries: "nothing inside" sits above every bin, "everything inside" below every bin
+        sh_bin[threadIdx.x] = (qq.trivial == 2u) ? -1 : (qq.trivial ? kBins1 : (int)(qq.prefix >> 16));
+        sh_slot[threadIdx.x] = qq.slot;
+    }
+    __syncthreads();
+    uint8_t* tab = table1 + (int64_t)m * kBins1;
+    for (int i = 0; i < per; ++i) {
+        const int b = b0 + i;
+        uint32_t code = 0;
+        for (int j = 0; j < nq; ++j) {
+            if (sh_bin[j] > b) ++code;
+            else if (sh_bin[j] == b) { code = 64u + sh_slot[j]; break; }
+            else break;  // bins are non-increasing in j
+        }
+        tab[b] = (uint8_t)code;
     }
 }
 
 // -------------------------------------------------------------------------------------------
-// digit passes 2 and 3 (fp32): histogram of the next 8 bits over the elements of the boundary bins
+// sweep 2 (fp32): per-interval energy of the bins that hold no threshold, and compaction of the keys
+// of the bins that do ("candidates": a few percent of the data) for the remaining digit passes
+// -------------------------------------------------------------------------------------------
+constexpr int kS2Threads = 256;
+constexpr int kS2Vecs = 4;                                   // 16-byte vectors per thread per round
+constexpr int kS2Round = kS2Threads * kS2Vecs * 4;            // elements per round
+constexpr int kStage = 2 * kS2Round;                          // staged candidate keys per block
+
+template <bool SUMS>
+__global__ void __launch_bounds__(kS2Threads)
+sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table1, int L,
+                       double* __restrict__ sum_partial, int sum_ctas, uint32_t* __restrict__ cand_keys,
+                       int64_t cand_cap, uint32_t* cand_count, int* cand_overflow, const int* worker_err) {
+    extern __shared__ __align__(16) uint8_t sh_raw[];
+    uint8_t* sh_table = sh_raw;                                                   // [32768]
+    uint32_t* sh_stage = reinterpret_cast<uint32_t*>(sh_raw + kBins1);            // [kStage]
+    double* sh_acc = reinterpret_cast<double*>(sh_raw + kBins1 + kStage * 4);     // [L][kS2Threads]
+    __shared__ uint32_t sh_n;
+    __shared__ uint32_t sh_base;
+    const int m = blockIdx.y;
+    if (worker_err[m]) return;
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(table1 + (int64_t)m * kBins1);
+        uint4* dst = reinterpret_cast<uint4*>(sh_table);
+        for (int i = threadIdx.x; i < kBins1 / 16; i += kS2Threads) dst[i] = src[i];
+        if (SUMS)
+            for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_acc[i] = 0.0;
+        if (threadIdx.x == 0) sh_n = 0;
+    }
+    __syncthreads();
+    const float* row = g + (int64_t)m * ld;
+    uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
+    int64_t v0, v1;
+    block_vector_range(d, 4, blockIdx.x, gridDim.x, &v0, &v1);
+
+    auto flush = [&]() {  // called by all threads
+        const uint32_t n = sh_n;
+        if (threadIdx.x == 0 && n) sh_base = atomicAdd(&cand_count[m], n);
+        __syncthreads();
+        if (n) {
+            const uint32_t base = sh_base;
+            if ((int64_t)base + n <= cand_cap) {
+                for (uint32_t i = threadIdx.x; i < n; i += kS2Threads) cand[base + i] = sh_stage[i];
+            } else if (threadIdx.x == 0) {
+                cand_overflow[m] = 1;  // too many keys share the boundary bins: the full-sweep passes take over
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) sh_n = 0;
+        __syncthreads();
+    };
+
+    for (int64_t vb = v0; vb < v1; vb += kS2Threads * kS2Vecs) {
+        uint4 q[kS2Vecs];
+        bool full[kS2Vecs];
+#pragma unroll
+        for (int j = 0; j < kS2Vecs; ++j) {
+            const int64_t v = vb + j * kS2Threads + threadIdx.x;
+            full[j] = (v < v1) && (v * 4 + 4 <= d);
+            if (full[j]) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v);
+        }
+#pragma unroll
+        for (int j = 0; j < kS2Vecs; ++j) {
+            const int64_t v = vb + j * kS2Threads + threadIdx.x;
+            uint32_t bits[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+            int cnt = full[j] ? 4 : 0;
+            if (!full[j] && v < v1) {  // ragged tail of the row
+                cnt = (int)(d - v * 4);
+                for (int c = 0; c < cnt; ++c) bits[c] = reinterpret_cast<const uint32_t*>(row)[v * 4 + c];
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (c < cnt) {
+                    const uint32_t key = bits[c] & 0x7FFFFFFFu;
+                    const uint32_t code = sh_table[key >> 16];
+                    if (code < 64u) {
+                        if (SUMS) {
+                            const double x = (double)__uint_as_float(key);
+                            double* a = &sh_acc[code * kS2Threads + threadIdx.x];
+                            *a = fma(x, x, *a);
+                        }
+                    } else {
+                        sh_stage[atomicAdd(&sh_n, 1u)] = key;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (sh_n > (uint32_t)(kStage - kS2Round)) flush();  // uniform: sh_n is read after the barrier
+    }
+    flush();
+    if (SUMS) {
+        for (int l = 0; l < L; ++l) {  // fixed-order tree: reproducible sums
+            double* a = sh_acc + l * kS2Threads;
+            for (int s = kS2Threads >> 1; s > 0; s >>= 1) {
+                if (threadIdx.x < s) a[threadIdx.x] += a[threadIdx.x + s];
+                __syncthreads();
+            }
+            if (threadIdx.x == 0) sum_partial[((int64_t)m * sum_ctas + blockIdx.x) * kMaxLevels + l] = a[0];
+        }
+    }
+}
+
+// Digit pass over the compacted candidate keys (normal case).
+template <int PASS>
+__global__ void __launch_bounds__(kSweepThreads)
+cand_pass_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const uint32_t* __restrict__ cand_count,
+                 const int* __restrict__ cand_overflow, const uint8_t* __restrict__ table1,
+                 const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err) {
+    __shared__ uint32_t sh_hist[kMaxQueries * kBins23];
+    const int m = blockIdx.y;
+    if (worker_err[m] || cand_overflow[m]) return;
+    const uint32_t n = cand_count[m];
+    if ((uint64_t)blockIdx.x * kSweepThreads >= n) return;
+    for (int i = threadIdx.x; i < kMaxQueries * kBins23; i += blockDim.x) sh_hist[i] = 0;
+    __syncthreads();
+    const uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
+    const uint8_t* tab = table1 + (int64_t)m * kBins1;
+    const uint8_t* mp = map2 + (int64_t)m * kMaxQueries * kBins23;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const uint32_t key = cand[i];
+        const uint32_t s2 = (uint32_t)__ldg(&tab[key >> 16]) - 64u;
+        if (PASS == 2) {
+            atomicAdd(&sh_hist[s2 * kBins23 + ((key >> 8) & 0xFFu)], 1u);
+        } else {
+            const uint32_t s3 = __ldg(&mp[s2 * kBins23 + ((key >> 8) & 0xFFu)]);
+            if (s3 != kNoSlot) atomicAdd(&sh_hist[s3 * kBins23 + (key & 0xFFu)], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t* out = hist_out + (int64_t)m * kMaxQueries * kBins23;
+    for (int i = threadIdx.x; i < kMaxQueries * kBins23; i += blockDim.x) {
+        const uint32_t c = sh_hist[i];
+        if (c) atomicAdd(&out[i], c);
+    }
+}
+
+// Energy of the candidate keys per open interval, now that the thresholds are exact.
+__global__ void __launch_bounds__(kS2Threads)
+cand_sums_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const uint32_t* __restrict__ cand_count,
+                 const int* __restrict__ cand_overflow, const Query* __restrict__ queries, int L,
+                 double* __restrict__ cand_partial, int cand_ctas, const int* worker_err) {
+    extern __shared__ double sh_acc2[];  // [L][kS2Threads]
+    __shared__ uint32_t sh_thr[kMaxQueries];
+    const int m = blockIdx.y;
+    if (worker_err[m] || cand_overflow[m]) return;
+    for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_acc2[i] = 0.0;
+    if (threadIdx.x < kMaxQueries)
+        sh_thr[threadIdx.x] = (threadIdx.x < L - 1) ? queries[m * kMaxQueries + threadIdx.x].T : 0u;
+    __syncthreads();
+    const uint32_t n = cand_count[m];
+    const uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
+    const int nthr = L - 1;
+    for (uint32_t i = blockIdx.x * kS2Threads + threadIdx.x; i < n; i += gridDim.x * kS2Threads) {
+        const uint32_t key = cand[i];
+        int lo = 0, hi = nthr;  // thresholds are descending: first index with T <= key
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (sh_thr[mid] > key) lo = mid + 1; else hi = mid;
+        }
+        if (lo == nthr || sh_thr[lo] != key) {
+            const double x = (double)__uint_as_float(key);
+            double* a = &sh_acc2[lo * kS2Threads + threadIdx.x];
+            *a = fma(x, x, *a);
+        }
+    }
+    __syncthreads();
+    for (int l = 0; l < L; ++l) {
+        double* a = sh_acc2 + l * kS2Threads;
+        for (int s = kS2Threads >> 1; s > 0; s >>= 1) {
+            if (threadIdx.x < s) a[threadIdx.x] += a[threadIdx.x + s];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) cand_partial[((int64_t)m * cand_ctas + blockIdx.x) * kMaxLevels + l] = a[0];
+    }
+}
+
+// -------------------------------------------------------------------------------------------
+// full-sweep digit passes (fp32): only for a worker whose candidate buffer overflowed, i.e. when a
+// large share of its entries falls into the boundary bins (many equal magnitudes)
 // -------------------------------------------------------------------------------------------
 template <int PASS>
 __global__ void __launch_bounds__(kSweepThreads)
 masked_pass_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table1,
-                   const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err) {
+                   const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err,
+                   const int* __restrict__ cand_overflow) {
     extern __shared__ uint8_t sh_raw[];
     uint32_t* sh_hist = reinterpret_cast<uint32_t*>(sh_raw);                        // [32][256]
     uint8_t* sh_table = sh_raw + kMaxQueries * kBins23 * sizeof(uint32_t);          // [32768]
     uint8_t* sh_map = sh_table + kBins1;                                            // [32][256] (pass 3)
     const int m = blockIdx.y;
-    if (worker_err[m]) return;
+    if (worker_err[m] || !cand_overflow[m]) return;
     for (int i = threadIdx.x; i < kMaxQueries * kBins23; i += blockDim.x) sh_hist[i] = 0;
     {
         const uint4* src = reinterpret_cast<const uint4*>(table1 + (int64_t)m * kBins1);
@@ -241,8 +441,9 @@ masked_pass_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uin
     for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
         for_each_in_vector<float>(row, v, d, [&](int64_t, uint32_t bits) {
             const uint32_t key = bits & 0x7FFFFFFFu;
-            const uint32_t s2 = sh_table[key >> 16];
-            if (s2 != kNoSlot) {
+            const uint32_t code = sh_table[key >> 16];
+            if (code >= 64u) {
+                const uint32_t s2 = code - 64u;
                 if (PASS == 2) {
                     atomicAdd(&sh_hist[s2 * kBins23 + ((key >> 8) & 0xFFu)], 1u);
                 } else {
@@ -315,7 +516,8 @@ resolve23_kernel(const uint32_t* hist, Query* queries, uint8_t* map2, int nq, co
 }
 
 // -------------------------------------------------------------------------------------------
-// band norms (adaptive): sum of g^2 over the open key intervals between consecutive thresholds
+// band norms by a full sweep (adaptive fp32, only for a worker whose candidate buffer overflowed):
+// sum of g^2 over the open key intervals between consecutive thresholds
 // -------------------------------------------------------------------------------------------
 // Element with key x belongs to open interval b = #{ l : T_l > x } unless x equals a threshold
 // (equal-key elements are split between bands by rank; their energy is added from the counts).
@@ -323,11 +525,12 @@ resolve23_kernel(const uint32_t* hist, Query* queries, uint8_t* map2, int nq, co
 // fixed reduction order, so the sums are reproducible.
 __global__ void __launch_bounds__(kSweepThreads)
 norm_sweep_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const Query* __restrict__ queries, int L,
-                  double* __restrict__ band_partial, int norm_ctas, const int* worker_err) {
+                  double* __restrict__ band_partial, int norm_ctas, const int* worker_err,
+                  const int* __restrict__ cand_overflow) {
     extern __shared__ double sh_acc[];  // [L][blockDim]
     __shared__ uint32_t sh_thr[kMaxQueries];
     const int m = blockIdx.y;
-    if (worker_err[m]) return;
+    if (worker_err[m] || !cand_overflow[m]) return;
     const int nt = blockDim.x;
     for (int i = threadIdx.x; i < L * nt; i += nt) sh_acc[i] = 0.0;
     if (threadIdx.x < kMaxQueries)
@@ -455,7 +658,10 @@ __device__ void fail_worker(int m, EmitParams* emit, int64_t* out_count, int32_t
 // |ranks of K  intersect  (k_{l-1}, k_l]| * val(K)^2;  Delta_l = sqrt(E_l);  p_l = Delta_l / sum Delta
 // (Lemma 3.4).  Then the level draw and the two thresholds of the drawn band.
 __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L, int64_t d, int is_bf16,
-                                  const double* band_partial, int n_partials, int norm_ctas, int adaptive,
+                                  const double* band_partial, int norm_ctas, int n_band,
+                                  const double* sum_partial, int sum_ctas, int n_sum,
+                                  const double* cand_partial, int cand_ctas, int n_cand,
+                                  const int* cand_overflow, int adaptive,
                                   uint64_t seed, uint64_t step, double* p_all, double* delta_all, double* u_dev,
                                   EmitParams* emit, int64_t* out_count, int32_t* out_level, double* out_p_sel,
                                   int64_t capacity, int* status, int* worker_err, int want_emit) {
@@ -469,8 +675,16 @@ __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L,
     }
     const int l = threadIdx.x;
     if (adaptive && l < L) {
+        // open-interval energy: per-block partials added in block order (reproducible).
+        // bf16 / overflowed fp32 worker: one source (histogram counts / full norm sweep);
+        // fp32 normal case: threshold-free bins from sweep 2 plus the candidate keys.
         double E = 0.0;
-        for (int c = 0; c < n_partials; ++c) E += band_partial[((int64_t)m * norm_ctas + c) * kMaxLevels + l];
+        if (is_bf16 || cand_overflow[m]) {
+            for (int c = 0; c < n_band; ++c) E += band_partial[((int64_t)m * norm_ctas + c) * kMaxLevels + l];
+        } else {
+            for (int c = 0; c < n_sum; ++c) E += sum_partial[((int64_t)m * sum_ctas + c) * kMaxLevels + l];
+            for (int c = 0; c < n_cand; ++c) E += cand_partial[((int64_t)m * cand_ctas + c) * kMaxLevels + l];
+        }
         const int64_t lo = l ? k[l - 1] : 0, hi = k[l];
         for (int j = 0; j < L - 1; ++j) {
             if (q[j].trivial) continue;
@@ -575,27 +789,66 @@ void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int
 }
 
 void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
-    if (dtype != MLMC_BF16) cudaMemsetAsync(ws.table1, 0xFF, (size_t)M * kBins1, s);
     LaunchScope t(ws, K_RESOLVE1, s);
     resolve1_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, ws.table1, L - 1, dtype == MLMC_BF16,
                                                   ws.worker_err);
 }
 
-void launch_masked_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s) {
+static int cand_blocks(const Workspace& ws, int M) {
+    int nb = (ws.sm_count * 2 + M - 1) / M;
+    if (nb > ws.cand_ctas) nb = ws.cand_ctas;
+    return nb < 1 ? 1 : nb;
+}
+
+// Sweep 2: energies of the threshold-free bins (adaptive only) and the candidate keys of the boundary bins.
+void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,
+                            cudaStream_t s) {
+    cudaMemsetAsync(ws.cand_count, 0, sizeof(uint32_t) * M, s);
+    cudaMemsetAsync(ws.cand_overflow, 0, sizeof(int) * M, s);
+    int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, 4);
+    if (nb > ws.sum_ctas) nb = ws.sum_ctas;
+    ws.cur_sum_ctas = nb;
+    const size_t smem = kBins1 + (size_t)kStage * 4 + (sums ? (size_t)L * kS2Threads * sizeof(double) : 0);
+    LaunchScope t(ws, K_SUMS_CAND, s);
+    if (sums)
+        sums_candidates_kernel<true><<<dim3(nb, M), kS2Threads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys, ws.cand_cap,
+            ws.cand_count, ws.cand_overflow, ws.worker_err);
+    else
+        sums_candidates_kernel<false><<<dim3(nb, M), kS2Threads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys, ws.cand_cap,
+            ws.cand_count, ws.cand_overflow, ws.worker_err);
+}
+
+// Digit pass 2 or 3: over the candidate keys, and (early exit unless the buffer overflowed) over the full row.
+void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s) {
     const size_t hist_bytes = (size_t)M * kMaxQueries * kBins23 * sizeof(uint32_t);
     const size_t smem = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
-    const int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 6);
+    const int nb_full = blocks_per_worker(ws, d, 4, kSweepThreads, M, 6);
+    const int nb_cand = cand_blocks(ws, M);
     if (pass == 2) {
         cudaMemsetAsync(ws.hist2, 0, hist_bytes, s);
         cudaMemsetAsync(ws.map2, 0xFF, (size_t)M * kMaxQueries * kBins23, s);
+        {
+            LaunchScope t(ws, K_CAND2, s);
+            cand_pass_kernel<2><<<dim3(nb_cand, M), kSweepThreads, 0, s>>>(ws.cand_keys, ws.cand_cap, ws.cand_count,
+                                                                           ws.cand_overflow, ws.table1, ws.map2,
+                                                                           ws.hist2, ws.worker_err);
+        }
         LaunchScope t(ws, K_MASKED2, s);
-        masked_pass_kernel<2><<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.table1,
-                                                                       ws.map2, ws.hist2, ws.worker_err);
+        masked_pass_kernel<2><<<dim3(nb_full, M), kSweepThreads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, ws.map2, ws.hist2, ws.worker_err, ws.cand_overflow);
     } else {
         cudaMemsetAsync(ws.hist3, 0, hist_bytes, s);
+        {
+            LaunchScope t(ws, K_CAND3, s);
+            cand_pass_kernel<3><<<dim3(nb_cand, M), kSweepThreads, 0, s>>>(ws.cand_keys, ws.cand_cap, ws.cand_count,
+                                                                           ws.cand_overflow, ws.table1, ws.map2,
+                                                                           ws.hist3, ws.worker_err);
+        }
         LaunchScope t(ws, K_MASKED3, s);
-        masked_pass_kernel<3><<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.table1,
-                                                                       ws.map2, ws.hist3, ws.worker_err);
+        masked_pass_kernel<3><<<dim3(nb_full, M), kSweepThreads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, ws.map2, ws.hist3, ws.worker_err, ws.cand_overflow);
     }
 }
 
@@ -607,17 +860,28 @@ void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
         resolve23_kernel<3><<<M, kResolveThreads, 0, s>>>(ws.hist3, ws.queries, ws.map2, L - 1, ws.worker_err);
 }
 
-void launch_norm_sweep(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
+// Band energies of the boundary bins from the candidate keys, and the full-sweep fallback.
+void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
+    {
+        const int nb = cand_blocks(ws, M);
+        ws.cur_cand_ctas = nb;
+        LaunchScope t(ws, K_CAND_SUMS, s);
+        cand_sums_kernel<<<dim3(nb, M), kS2Threads, (size_t)L * kS2Threads * sizeof(double), s>>>(
+            ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.queries, L, ws.cand_partial, ws.cand_ctas,
+            ws.worker_err);
+    }
     int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 4);
     if (nb > ws.norm_ctas) nb = ws.norm_ctas;
+    ws.cur_norm_ctas = nb;
     const size_t smem = (size_t)L * kSweepThreads * sizeof(double);
-    cudaMemsetAsync(ws.band_partial, 0, (size_t)M * ws.norm_ctas * kMaxLevels * sizeof(double), s);
     LaunchScope t(ws, K_NORM_SWEEP, s);
     norm_sweep_kernel<<<dim3(nb, M), kSweepThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.queries, L,
-                                                               ws.band_partial, ws.norm_ctas, ws.worker_err);
+                                                               ws.band_partial, ws.norm_ctas, ws.worker_err,
+                                                               ws.cand_overflow);
 }
 
 void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s) {
+    ws.cur_norm_ctas = 1;
     LaunchScope t(ws, K_NORM_HIST, s);
     norm_from_hist_bf16_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, L, ws.band_partial, ws.norm_ctas,
                                                              ws.worker_err);
@@ -625,12 +889,13 @@ void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s) {
 
 void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool adaptive, bool want_emit,
                        uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, cudaStream_t s) {
-    const int n_partials = (dtype == MLMC_BF16) ? 1 : ws.norm_ctas;
     LaunchScope t(ws, K_PROBS_DRAW, s);
     probs_draw_kernel<<<M, kMaxLevels, 0, s>>>(
-        ws.queries, ws.k_dev, L, d, dtype == MLMC_BF16, ws.band_partial, n_partials, ws.norm_ctas, adaptive ? 1 : 0,
-        seed, step, ws.p_all, ws.delta_all, ws.u_dev, ws.emit, out ? out->count : nullptr, out ? out->level : nullptr,
-        out ? out->p_sel : nullptr, out ? out->capacity : 0, ws.status, ws.worker_err, want_emit ? 1 : 0);
+        ws.queries, ws.k_dev, L, d, dtype == MLMC_BF16, ws.band_partial, ws.norm_ctas, ws.cur_norm_ctas,
+        ws.sum_partial, ws.sum_ctas, ws.cur_sum_ctas, ws.cand_partial, ws.cand_ctas, ws.cur_cand_ctas,
+        ws.cand_overflow, adaptive ? 1 : 0, seed, step, ws.p_all, ws.delta_all, ws.u_dev, ws.emit,
+        out ? out->count : nullptr, out ? out->level : nullptr, out ? out->p_sel : nullptr, out ? out->capacity : 0,
+        ws.status, ws.worker_err, want_emit ? 1 : 0);
 }
 
 void launch_copy_probs(Workspace& ws, int M, int L, const double* p_fixed, double* p_out, double* delta_out,
@@ -654,6 +919,14 @@ int configure_select_kernels() {
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     e = cudaFuncSetAttribute(norm_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxLevels * kSweepThreads * sizeof(double)));
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    const int smem_s2 = kBins1 + kStage * 4 + kMaxLevels * kS2Threads * (int)sizeof(double);
+    e = cudaFuncSetAttribute(sums_candidates_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    e = cudaFuncSetAttribute(sums_candidates_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    e = cudaFuncSetAttribute(cand_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kMaxLevels * kS2Threads * sizeof(double)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     return MLMC_OK;
 }

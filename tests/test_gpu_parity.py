@@ -214,6 +214,19 @@ def test_topk_degenerate_inputs(B, ora, ctx, case):
             check_topk(B, ora, ctx, gb, k, None, 10, step, expect_excluded=1)
 
 
+def test_topk_candidate_overflow_takes_the_full_sweep_path(B, ora, ctx):
+    # Nearly all entries share two magnitudes, so the boundary bins hold more keys than the candidate
+    # buffer of this context (2^20 per worker): the digit passes and the band norms fall back to full sweeps.
+    rng = np.random.default_rng(25)
+    d = 1_300_000
+    g_np = rng.choice(np.array([0.5, -0.5, 0.5000001, 3.0], dtype=np.float32), (2, d), p=[0.4, 0.3, 0.29, 0.01])
+    g = to_dev(g_np)
+    k = [100, 20_000, 400_000, 900_000, d]
+    for step in range(3):
+        check_topk(B, ora, ctx, g, k, None, 11, step, expect_excluded=1)
+        check_topk(B, ora, ctx, g, k, list(wl.geometric_probs(len(k))), 11, step)
+
+
 def test_topk_single_level_is_identity(B, ora, ctx):
     g_np = np.random.default_rng(23).standard_normal((3, 4097)).astype(np.float32)
     g = to_dev(g_np)
