@@ -139,8 +139,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     for (int i = 0; i < K_COUNT; ++i) ws.launches_by_id[i] = 0;
     ws.norm_ctas = ws.sm_count * 4;
     ws.sum_ctas = ws.sm_count * 4;
-    ws.cand_ctas = ws.sm_count * 2;
-    ws.cur_norm_ctas = ws.cur_sum_ctas = ws.cur_cand_ctas = 0;
+    ws.cur_norm_ctas = ws.cur_sum_ctas = 0;
     // candidate keys: a quarter of the row (boundary bins normally hold a few percent of it); small rows fit whole
     ws.cand_cap = d_max / 4 > (int64_t(1) << 20) ? d_max / 4 : (d_max < (int64_t(1) << 20) ? d_max : (int64_t(1) << 20));
     ws.stat_ctas = ws.sm_count * 4;
@@ -159,7 +158,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_queries = pl.take(sizeof(Query) * kMaxQueries * M_max);
     const size_t o_band = pl.take(sizeof(double) * kMaxLevels * ws.norm_ctas * M_max);
     const size_t o_sum = pl.take(sizeof(double) * kMaxLevels * ws.sum_ctas * M_max);
-    const size_t o_cpart = pl.take(sizeof(double) * kMaxLevels * ws.cand_ctas * M_max);
+    const size_t o_cpart = pl.take(sizeof(unsigned long long) * kMaxLevels * 4 * M_max);
     const size_t o_ckeys = pl.take(sizeof(uint32_t) * ws.cand_cap * M_max);
     const size_t o_ccount = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_cover = pl.take(sizeof(int) * M_max);
@@ -198,7 +197,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.queries = reinterpret_cast<Query*>(base + o_queries);
     ws.band_partial = reinterpret_cast<double*>(base + o_band);
     ws.sum_partial = reinterpret_cast<double*>(base + o_sum);
-    ws.cand_partial = reinterpret_cast<double*>(base + o_cpart);
+    ws.cand_S = reinterpret_cast<unsigned long long*>(base + o_cpart);
     ws.cand_keys = reinterpret_cast<uint32_t*>(base + o_ckeys);
     ws.cand_count = reinterpret_cast<uint32_t*>(base + o_ccount);
     ws.cand_overflow = reinterpret_cast<int*>(base + o_cover);

@@ -81,8 +81,7 @@ struct Workspace {
     int norm_ctas, cur_norm_ctas;
     double* sum_partial;         // [M][sum_ctas][kMaxLevels]  sweep 2: energy of the threshold-free bins
     int sum_ctas, cur_sum_ctas;
-    double* cand_partial;        // [M][cand_ctas][kMaxLevels] energy of the candidate keys
-    int cand_ctas, cur_cand_ctas;
+    unsigned long long* cand_S;  // [M][kMaxLevels][2 sides][2 halves] integer energy sums of the candidate keys
     uint32_t* cand_keys;         // [M][cand_cap] keys of the boundary-bin elements
     int64_t cand_cap;
     uint32_t* cand_count;        // [M]

@@ -368,22 +368,31 @@ cand_pass_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const
 }
 
 // Energy of the candidate keys per open interval, now that the thresholds are exact.
-__global__ void __launch_bounds__(kS2Threads)
+// The candidate buffer is filled in an order that changes from run to run, so the sums are taken in
+// integers, where the order does not matter: every candidate lies in a boundary bin, all keys of one
+// bin share their exponent, so g^2 = mant^2 * 2^(2 (max(e,1) - 150)) with a 48-bit integer mant^2.
+// An open interval (T_l, T_{l-1}) meets at most two boundary bins: the bin of T_{l-1} (side 0) and
+// the bin of T_l (side 1).  Per (interval, side) the low and the high 24 bits of mant^2 are added
+// separately in u64 (no overflow below 2^40 terms) and combined in 128 bits by the draw kernel.
+constexpr int kCandSumThreads = 128;
+
+__global__ void __launch_bounds__(kCandSumThreads)
 cand_sums_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const uint32_t* __restrict__ cand_count,
                  const int* __restrict__ cand_overflow, const Query* __restrict__ queries, int L,
-                 double* __restrict__ cand_partial, int cand_ctas, const int* worker_err) {
-    extern __shared__ double sh_acc2[];  // [L][kS2Threads]
+                 unsigned long long* __restrict__ cand_S, const int* worker_err) {
+    extern __shared__ unsigned long long sh_S[];  // [L][4][kCandSumThreads]: (side, half) pairs per interval
     __shared__ uint32_t sh_thr[kMaxQueries];
     const int m = blockIdx.y;
     if (worker_err[m] || cand_overflow[m]) return;
-    for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_acc2[i] = 0.0;
+    const uint32_t n = cand_count[m];
+    if ((uint64_t)blockIdx.x * kCandSumThreads >= n) return;
+    for (int i = threadIdx.x; i < L * 4 * kCandSumThreads; i += kCandSumThreads) sh_S[i] = 0ull;
     if (threadIdx.x < kMaxQueries)
         sh_thr[threadIdx.x] = (threadIdx.x < L - 1) ? queries[m * kMaxQueries + threadIdx.x].T : 0u;
     __syncthreads();
-    const uint32_t n = cand_count[m];
     const uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
     const int nthr = L - 1;
-    for (uint32_t i = blockIdx.x * kS2Threads + threadIdx.x; i < n; i += gridDim.x * kS2Threads) {
+    for (uint32_t i = blockIdx.x * kCandSumThreads + threadIdx.x; i < n; i += gridDim.x * kCandSumThreads) {
         const uint32_t key = cand[i];
         int lo = 0, hi = nthr;  // thresholds are descending: first index with T <= key
         while (lo < hi) {
@@ -391,19 +400,23 @@ cand_sums_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const
             if (sh_thr[mid] > key) lo = mid + 1; else hi = mid;
         }
         if (lo == nthr || sh_thr[lo] != key) {
-            const double x = (double)__uint_as_float(key);
-            double* a = &sh_acc2[lo * kS2Threads + threadIdx.x];
-            *a = fma(x, x, *a);
+            const int side = (lo > 0 && (sh_thr[lo - 1] >> 16) == (key >> 16)) ? 0 : 1;
+            const uint64_t mant = (key & 0x7FFFFFu) | ((key >> 23) ? 0x800000u : 0u);
+            const uint64_t m2 = mant * mant;
+            unsigned long long* a = &sh_S[((lo * 2 + side) * 2) * kCandSumThreads + threadIdx.x];
+            a[0] += m2 & 0xFFFFFFull;
+            a[kCandSumThreads] += m2 >> 24;
         }
     }
     __syncthreads();
-    for (int l = 0; l < L; ++l) {
-        double* a = sh_acc2 + l * kS2Threads;
-        for (int s = kS2Threads >> 1; s > 0; s >>= 1) {
+    unsigned long long* out = cand_S + (int64_t)m * kMaxLevels * 4;
+    for (int q = 0; q < L * 4; ++q) {
+        unsigned long long* a = sh_S + q * kCandSumThreads;
+        for (int s = kCandSumThreads >> 1; s > 0; s >>= 1) {
             if (threadIdx.x < s) a[threadIdx.x] += a[threadIdx.x + s];
             __syncthreads();
         }
-        if (threadIdx.x == 0) cand_partial[((int64_t)m * cand_ctas + blockIdx.x) * kMaxLevels + l] = a[0];
+        if (threadIdx.x == 0 && a[0]) atomicAdd(&out[q], a[0]);  // integer: the order of the blocks does not matter
     }
 }
 
@@ -660,7 +673,7 @@ __device__ void fail_worker(int m, EmitParams* emit, int64_t* out_count, int32_t
 __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L, int64_t d, int is_bf16,
                                   const double* band_partial, int norm_ctas, int n_band,
                                   const double* sum_partial, int sum_ctas, int n_sum,
-                                  const double* cand_partial, int cand_ctas, int n_cand,
+                                  const unsigned long long* cand_S,
                                   const int* cand_overflow, int adaptive,
                                   uint64_t seed, uint64_t step, double* p_all, double* delta_all, double* u_dev,
                                   EmitParams* emit, int64_t* out_count, int32_t* out_level, double* out_p_sel,
@@ -683,7 +696,17 @@ __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L,
             for (int c = 0; c < n_band; ++c) E += band_partial[((int64_t)m * norm_ctas + c) * kMaxLevels + l];
         } else {
             for (int c = 0; c < n_sum; ++c) E += sum_partial[((int64_t)m * sum_ctas + c) * kMaxLevels + l];
-            for (int c = 0; c < n_cand; ++c) E += cand_partial[((int64_t)m * cand_ctas + c) * kMaxLevels + l];
+            // candidate keys of the two boundary bins that meet this interval: exact integer sums of mant^2
+            for (int side = 0; side < 2; ++side) {
+                const unsigned long long* S = cand_S + ((int64_t)m * kMaxLevels + l) * 4 + side * 2;
+                const int j = side ? l : l - 1;  // the threshold whose bin fixes the exponent
+                if ((S[0] | S[1]) && j >= 0 && j < L - 1) {
+                    const int e = (int)(q[j].T >> 23);
+                    const unsigned __int128 tot = ((unsigned __int128)S[1] << 24) + S[0];
+                    const double td = (double)(unsigned long long)(tot >> 64) * 0x1.0p64 + (double)(unsigned long long)tot;
+                    E += ldexp(td, 2 * ((e ? e : 1) - 150));
+                }
+            }
         }
         const int64_t lo = l ? k[l - 1] : 0, hi = k[l];
         for (int j = 0; j < L - 1; ++j) {
@@ -796,7 +819,6 @@ void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
 
 static int cand_blocks(const Workspace& ws, int M) {
     int nb = (ws.sm_count * 2 + M - 1) / M;
-    if (nb > ws.cand_ctas) nb = ws.cand_ctas;
     return nb < 1 ? 1 : nb;
 }
 
@@ -864,11 +886,10 @@ void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
 void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
     {
         const int nb = cand_blocks(ws, M);
-        ws.cur_cand_ctas = nb;
+        cudaMemsetAsync(ws.cand_S, 0, (size_t)M * kMaxLevels * 4 * sizeof(unsigned long long), s);
         LaunchScope t(ws, K_CAND_SUMS, s);
-        cand_sums_kernel<<<dim3(nb, M), kS2Threads, (size_t)L * kS2Threads * sizeof(double), s>>>(
-            ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.queries, L, ws.cand_partial, ws.cand_ctas,
-            ws.worker_err);
+        cand_sums_kernel<<<dim3(nb, M), kCandSumThreads, (size_t)L * 4 * kCandSumThreads * sizeof(unsigned long long), s>>>(
+            ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.queries, L, ws.cand_S, ws.worker_err);
     }
     int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 4);
     if (nb > ws.norm_ctas) nb = ws.norm_ctas;
@@ -892,7 +913,7 @@ void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool a
     LaunchScope t(ws, K_PROBS_DRAW, s);
     probs_draw_kernel<<<M, kMaxLevels, 0, s>>>(
         ws.queries, ws.k_dev, L, d, dtype == MLMC_BF16, ws.band_partial, ws.norm_ctas, ws.cur_norm_ctas,
-        ws.sum_partial, ws.sum_ctas, ws.cur_sum_ctas, ws.cand_partial, ws.cand_ctas, ws.cur_cand_ctas,
+        ws.sum_partial, ws.sum_ctas, ws.cur_sum_ctas, ws.cand_S,
         ws.cand_overflow, adaptive ? 1 : 0, seed, step, ws.p_all, ws.delta_all, ws.u_dev, ws.emit,
         out ? out->count : nullptr, out ? out->level : nullptr, out ? out->p_sel : nullptr, out ? out->capacity : 0,
         ws.status, ws.worker_err, want_emit ? 1 : 0);
@@ -926,7 +947,7 @@ int configure_select_kernels() {
     e = cudaFuncSetAttribute(sums_candidates_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     e = cudaFuncSetAttribute(cand_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(kMaxLevels * kS2Threads * sizeof(double)));
+                             (int)(kMaxLevels * 4 * kCandSumThreads * sizeof(unsigned long long)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     return MLMC_OK;
 }
