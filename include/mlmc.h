@@ -140,6 +140,28 @@ int mlmc_compress_bitwise(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, in
 int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, int L, int M, int64_t d,
                    float* out, void* stream);
 
+/* The Top-k case of mlmc_aggregate for callers that must not allocate device memory.  (The paper
+ * has no counterpart: this is a deployment variant of the same averaging step.)
+ *
+ * mlmc_aggregate keeps a small table of tile offsets in the workspace of an mlmc_ctx, and creating a
+ * context calls cudaMalloc.  Code that runs after a framework has claimed the whole GPU for its own
+ * memory pool, inside a region where the allocator may not be entered (a real-time loop, a callback
+ * from another library, a process whose memory budget is fixed at start-up), cannot do that.  This
+ * entry point needs no context: its table lives in a device array compiled into the library, 4 MiB
+ * that every GPU which loads the library holds until the process exits.  It calls neither cudaMalloc
+ * nor cudaFree nor any routine that allocates.
+ *
+ *   msgs, out   as for mlmc_aggregate with kind MLMC_TOPK: host struct of device pointers, dense out[d].
+ *   Limit       M * (ceil(d / 4096) + 1) <= 2^20; larger problems return MLMC_ERR_ARG and nothing is launched.
+ *   Device      the current device of the calling thread; msgs and out must live there.
+ *   First call  on each device looks up the device address of the built-in table (a synchronous
+ *               runtime query); make that first call before starting any stream capture.
+ *   Sharing     every call on a device uses the same table.  Each call rewrites all entries it reads,
+ *               so nothing carries over between calls, but two calls whose kernels overlap on the GPU
+ *               (different streams, or several host threads) race: run them one after the other.
+ * The result is identical to mlmc_aggregate's on the same messages. */
+int mlmc_aggregate_topk_noalloc(const mlmc_topk_msgs* msgs, int M, int64_t d, float* out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

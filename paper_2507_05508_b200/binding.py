@@ -24,7 +24,8 @@ MLMC_MAX_LEVELS = 32
 
 EXPORTS = ["mlmc_create", "mlmc_destroy", "mlmc_get_status", "mlmc_launch_count", "mlmc_read_u",
            "mlmc_kernel_count", "mlmc_kernel_name", "mlmc_timing_enable", "mlmc_timing_read",
-           "mlmc_level_probs", "mlmc_compress_topk", "mlmc_compress_bitwise", "mlmc_aggregate"]
+           "mlmc_level_probs", "mlmc_compress_topk", "mlmc_compress_bitwise", "mlmc_aggregate",
+           "mlmc_aggregate_topk_noalloc"]
 
 
 class MlmcError(RuntimeError):
@@ -65,6 +66,7 @@ def lib() -> C.CDLL:
         L.mlmc_compress_topk.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_compress_bitwise.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_aggregate.argtypes = [vp, i32, vp, vp, i32, i32, i64, vp, vp]
+        L.mlmc_aggregate_topk_noalloc.argtypes = [vp, i32, i64, vp, vp]
         L.mlmc_kernel_count.argtypes = []
         L.mlmc_kernel_name.argtypes = [i32]
         L.mlmc_timing_enable.argtypes = [vp, i32]
@@ -181,6 +183,13 @@ def mlmc_aggregate(ctx, kind: int, msgs, b: Optional[Sequence[int]], M: int, d: 
     bh = _host_array(C.c_int32, None if b is None else list(b))
     _check(lib().mlmc_aggregate(ctx, kind, C.byref(msgs.struct), bh, 0 if b is None else len(b), M, d,
                                 out.data_ptr(), _stream()), "mlmc_aggregate")
+
+
+def mlmc_aggregate_topk_noalloc(msgs: "TopkBuffers", M: int, d: int, out: torch.Tensor) -> None:
+    """Top-k server average that needs no context and allocates nothing (fixed built-in scratch; see mlmc.h)."""
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.numel() >= d
+    _check(lib().mlmc_aggregate_topk_noalloc(C.byref(msgs.struct), M, d, out.data_ptr(), _stream()),
+           "mlmc_aggregate_topk_noalloc")
 
 
 class TopkBuffers:

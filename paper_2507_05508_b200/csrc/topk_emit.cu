@@ -278,3 +278,57 @@ void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int
 }
 
 }  // namespace mlmc
+
+// ---------------------------------------------------------------------------------------------
+// Server average of Top-k messages without any allocation.
+// ---------------------------------------------------------------------------------------------
+// The tile offsets that the averaging kernel needs normally live in the context's workspace, which
+// mlmc_create obtains with cudaMalloc.  Here they live in a file-scope device array of fixed size,
+// which every GPU that loads this library holds until the process exits.
+namespace mlmc {
+namespace {
+
+constexpr int64_t kStaticOffsetWords = int64_t(1) << 20;  // 4 MiB: M * (ceil(d / kAggTile) + 1) entries at most
+static __device__ __align__(256) uint32_t g_static_offsets[kStaticOffsetWords];
+
+constexpr int kMaxDevices = 64;
+uint32_t* g_static_offsets_addr[kMaxDevices];  // device address of the array on each device, 0 = not looked up yet
+int g_static_sm_count[kMaxDevices];
+
+}  // namespace
+}  // namespace mlmc
+
+extern "C" int mlmc_aggregate_topk_noalloc(const mlmc_topk_msgs* msgs, int M, int64_t d, float* out, void* stream) {
+    using namespace mlmc;
+    if (!msgs || !out || !msgs->idx || !msgs->val || !msgs->count || !msgs->level) return MLMC_ERR_ARG;
+    if (M < 1 || d < 1 || d >= (int64_t(1) << 32) || msgs->capacity < 0) return MLMC_ERR_ARG;
+    const int64_t ntiles = (d + kAggTile - 1) / kAggTile;
+    const int64_t n_off = (int64_t)M * (ntiles + 1);
+    if (n_off > kStaticOffsetWords) return MLMC_ERR_ARG;  // beyond the fixed scratch: use mlmc_aggregate with a context
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MLMC_ERR_CUDA;
+    if (!g_static_offsets_addr[dev]) {
+        // Set-up, once per device, with that device current.  In host code the array's name only stands
+        // for the symbol; the address a kernel can use has to be asked for.
+        uint32_t* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_offsets) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return MLMC_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+            return MLMC_ERR_CUDA;
+        g_static_sm_count[dev] = sms;
+        g_static_offsets_addr[dev] = p;
+    }
+    uint32_t* offsets = g_static_offsets_addr[dev];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // every entry in [0, n_off) is rewritten by this kernel, so nothing is left over from an earlier call
+    agg_offsets_kernel<<<(unsigned)((n_off + 255) / 256), 256, 0, s>>>(msgs->idx, msgs->count, msgs->level,
+                                                                       msgs->capacity, M, (int)ntiles, offsets);
+    int64_t grid = (int64_t)g_static_sm_count[dev] * 8;
+    if (grid > ntiles) grid = ntiles;
+    aggregate_topk_kernel<<<(unsigned)grid, 256, 0, s>>>(msgs->idx, msgs->val, msgs->capacity, M, d, (int)ntiles,
+                                                         offsets, out);
+    return cudaGetLastError() == cudaSuccess ? MLMC_OK : MLMC_ERR_CUDA;
+}
