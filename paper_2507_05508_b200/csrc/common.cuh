@@ -16,9 +16,12 @@ constexpr uint32_t kKeyNone = 0xFFFFFFFFu;    // threshold above every finite ke
 constexpr uint32_t kNoSlot = 0xFFu;
 
 constexpr int kSweepThreads = 512;            // histogram / masked / norm sweeps
-constexpr int kEmitThreads = 128;
-constexpr int kEmitItems = 16;                // elements per thread per tile
-constexpr int kEmitTile = kEmitThreads * kEmitItems;
+constexpr int kEmitWorkers = 8;               // warps that count and write; one more warp per block computes the prefixes
+constexpr int kEmitThreads = (kEmitWorkers + 1) * 32;
+constexpr int kEmitBlocksPerSM = 3;
+constexpr int kEmitRows = 16;                 // 32-bit words per lane per tile (1 fp32 or 2 bf16 elements each)
+constexpr int kEmitStages = 4;                // tiles of one block resident in shared memory
+constexpr int kEmitTile = kEmitWorkers * 32 * kEmitRows;   // words per tile = elements per fp32 tile; bf16: twice as many
 constexpr int kAggTile = 4096;                // dense output elements per aggregation tile
 
 // Per-worker selection query: the rank-k element of the total order.
@@ -92,9 +95,9 @@ struct Workspace {
     double* delta_all;           // [M][kMaxLevels]
     double* u_dev;               // [M]
     EmitParams* emit;            // [M]
-    uint4* tile_desc;            // [max_tiles] look-back records {D, Ea, Eb, state}
+    uint4* tile_desc;            // [max_tiles] look-back records {C, A, B, state}
     int64_t max_tiles;
-    unsigned int* tile_counter;  // [M] ticket counters: tiles are numbered in the order they start
+    unsigned int* tile_counter;  // ticket counter (entry 0): tiles are numbered in the order they are taken
     uint32_t* agg_offsets;       // [M][agg_tiles_max + 1]
     // bit-wise
     uint32_t* gmax_bits;         // [M]
@@ -232,6 +235,7 @@ void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool a
 void launch_copy_probs(Workspace& ws, int M, int L, const double* p_fixed, double* p_out, double* delta_out,
                        cudaStream_t s);
 // topk_emit.cu
+int configure_emit_kernels();
 void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const mlmc_topk_msgs& out,
                  cudaStream_t s);
 void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int64_t d, float* out, cudaStream_t s);

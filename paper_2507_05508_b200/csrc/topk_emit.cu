@@ -4,7 +4,7 @@
 //   { i : k_{l-1} < rank(i) <= k_l },  as (i, g_i / p_l) in ascending i  (Eq. 5 with g^0 = 0; Alg. 2 "Send").
 // Membership is decided from the two thresholds (Ta, ra), (Tb, rb) of the band; equal-key elements
 // are admitted by their index-ordered rank, so the running counts
-//   D  = #{ Tb < key <= Ta },  Ea = #{ key == Ta },  Eb = #{ key == Tb }
+//   C = #{ Tb <= key <= Ta },  A = #{ key == Ta },  B = #{ key == Tb }
 // are carried across tiles with a decoupled look-back (tiles are numbered by a ticket counter, so
 // every predecessor of a running tile has already started; every wait is bounded).
 //
@@ -17,188 +17,487 @@ namespace mlmc {
 
 namespace {
 
-constexpr unsigned kSpinLimit = 1u << 22;  // polls before a look-back gives up (each poll is a global load)
+constexpr unsigned kSpinLimit = 1u << 22;          // polls of a shared-memory word before a wait gives up
+constexpr unsigned kLookbackSpinLimit = 1u << 20;  // polls of a look-back record (each poll is a global load)
+constexpr int kTicketRing = 8;
 
-// Look-back record of one tile: {D, Ea, Eb, state}, state 0 = not yet, 1 = the tile's own counts,
-// 2 = running totals up to and including the tile.  A record is written and read as one 16-byte
-// access, so counts and state always belong together.
-__device__ __forceinline__ void put_record(uint4* rec, uint32_t D, uint32_t Ea, uint32_t Eb, uint32_t state) {
-    __stcg(rec, make_uint4(D, Ea, Eb, state));
+// Look-back record of one tile: {C, A, B, state}: closed-range keys (Tb <= key <= Ta), keys equal to Ta,
+// keys equal to Tb; state 0 = not yet, 1 = the tile's own counts, 2 = running totals up to and including
+// the tile.  A record is written and read as one 16-byte access, so counts and state belong together.
+__device__ __forceinline__ void put_record(uint4* rec, uint32_t C, uint32_t A, uint32_t B, uint32_t state) {
+    __stcg(rec, make_uint4(C, A, B, state));
 }
 
-__device__ __forceinline__ uint32_t warp_sum(uint32_t x) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
-    return x;
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+    const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sa), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
-// One block per tile of kEmitTile consecutive entries of one worker (blockIdx.y).  Tiles are numbered by
-// a per-worker ticket taken when the block starts, so every lower-numbered tile is already running and
-// will publish its counts without waiting for anyone.
+// How a 32-bit word of the gradient row maps to elements: one fp32 element, or two bf16 elements
+// (low half first).  A word past the end of the row reads as kPad, whose keys lie above every
+// threshold the kernel uses (thresholds are clamped to kCap, the key of +Inf), so padded elements
+// are never inside the band.
 template <typename T>
-__global__ void __launch_bounds__(kEmitThreads, 10)
-emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker,
+struct EmitWord;
+
+template <>
+struct EmitWord<float> {
+    static constexpr int S = 1;
+    static constexpr uint32_t kPad = 0x7FFFFFFFu;
+    static constexpr uint32_t kCap = 0x7F800000u;
+    __device__ static __forceinline__ uint32_t key(uint32_t w, int) { return w & 0x7FFFFFFFu; }
+    __device__ static __forceinline__ float value(uint32_t w, int) { return __uint_as_float(w); }
+};
+
+template <>
+struct EmitWord<bf16_t> {
+    static constexpr int S = 2;
+    static constexpr uint32_t kPad = 0x7FFF7FFFu;
+    static constexpr uint32_t kCap = 0x7F80u;
+    __device__ static __forceinline__ uint32_t key(uint32_t w, int s) { return s ? ((w >> 16) & 0x7FFFu) : (w & 0x7FFFu); }
+    __device__ static __forceinline__ float value(uint32_t w, int s) {
+        return __uint_as_float(s ? (w & 0xFFFF0000u) : (w << 16));
+    }
+};
+
+// Number of band entries among a prefix of the row that holds C closed-range keys, A keys equal to Ta
+// and B keys equal to Tb: the first min(A, ra) ties of Ta belong to Top-k_{l-1} (not to the band), and
+// only the first min(B, rb) ties of Tb belong to Top-k_l.
+__device__ __forceinline__ uint32_t band_prefix(uint32_t C, uint32_t A, uint32_t B, uint32_t ra, uint32_t rb) {
+    return C - B + min(B, rb) - min(A, ra);
+}
+
+// Starts the copy of one warp's share (kEmitRows * 32 consecutive words) of tile t of a row into its
+// share of a shared-memory slot.  Full tiles go as 16-byte asynchronous copies; the ragged last tile of
+// a row is written with plain stores, padded with kPad.
+template <typename T>
+__device__ __forceinline__ void emit_fetch_share(const T* __restrict__ row, int64_t d, int64_t tile, uint32_t* share,
+                                                 int warp, int lane) {
+    using EW = EmitWord<T>;
+    constexpr int kShare = kEmitRows * 32;
+    const int64_t w0 = tile * kEmitTile + warp * kShare;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(row) + w0;
+    if ((tile + 1) * kEmitTile * EW::S <= d) {
+#pragma unroll
+        for (int c = lane; c < kShare / 4; c += 32) cp_async_16(share + c * 4, words + c * 4);
+    } else {
+        for (int i = lane; i < kShare; i += 32) {
+            const int64_t wi = w0 + i;
+            uint32_t v = EW::kPad;
+            if ((wi + 1) * EW::S <= d) {
+                v = __ldg(words + i);
+            } else if (EW::S == 2 && wi * 2 < d) {  // odd bf16 tail: only the low half exists
+                v = (uint32_t)reinterpret_cast<const uint16_t*>(row)[wi * 2] | 0x7FFF0000u;
+            }
+            share[i] = v;
+        }
+    }
+}
+
+// Block-local hand-over words between the worker warps and the prefix warp.  All counters only grow.
+struct EmitSync {
+    unsigned tickets_ready;         // tickets [0, tickets_ready) of this block are in the ticket ring
+    unsigned counted[kEmitStages];  // per slot: worker warps that have posted counts (kEmitWorkers more per tile;
+                                    // per slot, because a fast warp may count tile k+1 before a slow one counts tile k)
+    unsigned prefix_ready;          // tiles [0, prefix_ready) of this block have their prefix in shared memory
+    int abort;                      // a bounded wait gave up: everybody leaves
+};
+
+__device__ __forceinline__ unsigned ld_volatile_shared(const unsigned* p) { return *reinterpret_cast<const volatile unsigned*>(p); }
+
+// The whole warp spins until *p >= want (bounded).  Returns false, for every lane alike, when the wait
+// gave up (which raises the block's abort flag) or another warp had raised it.
+__device__ __forceinline__ bool wait_at_least(const unsigned* p, unsigned want, int* abort_flag) {
+    unsigned spins = 0;
+    bool ok = true;
+    while (ld_volatile_shared(p) < want) {
+        if (*reinterpret_cast<volatile int*>(abort_flag)) {
+            ok = false;
+            break;
+        }
+        if (++spins > kSpinLimit) {
+            *reinterpret_cast<volatile int*>(abort_flag) = 1;
+            ok = false;
+            break;
+        }
+    }
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    __threadfence_block();
+    return ok;
+}
+
+// Persistent blocks take tiles in ticket order; consecutive tickets go to different workers (ticket q is
+// tile q / M of worker q % M).  Eight worker warps each own a fixed share of every tile; a ninth warp
+// owns the tickets and the prefixes, so nobody waits at a block-wide barrier:
+//   worker, iteration k:  count its share of tile k (closed-range keys Tb <= key <= Ta, ties of Ta and Tb),
+//                         write its share of tile k-2 at the final positions (within a warp row the band
+//                         entries are consecutive, so the stores coalesce), start the copy of tile k+2;
+//   prefix warp, tile j:  when all shares of tile j are counted, publish the tile's counts; then finish
+//                         tile j-1: sum the records of the worker's earlier tiles (decoupled look-back)
+//                         and hand the prefix to the workers.
+// Every wait is bounded; a wait that gives up sets MLMC_ERR_TIMEOUT and makes the block leave.
+template <typename T>
+__global__ void __launch_bounds__(kEmitThreads, kEmitBlocksPerSM)
+emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker, unsigned total_tiles, int M,
             const EmitParams* __restrict__ emit, uint4* tile_desc, unsigned* tile_counter,
             uint32_t* __restrict__ idx_out, float* __restrict__ val_out, int64_t capacity, int* status,
             int* worker_err) {
-    using Tr = ElemTraits<T>;
-    constexpr int V = Tr::kVec;
-    constexpr int NV = kEmitItems / V;
-    constexpr int kWarps = kEmitThreads / 32;
-    __shared__ unsigned sh_ticket;
-    __shared__ unsigned long long sh_warp[kWarps];
-    __shared__ uint32_t sh_prefix[4];  // D, Ea, Eb, ok
+    using EW = EmitWord<T>;
+    constexpr int S = EW::S;
+    constexpr int kShare = kEmitRows * 32;
+    extern __shared__ __align__(16) uint32_t sh_ring[];  // [kEmitStages][kEmitTile]
+    __shared__ EmitSync sy;
+    __shared__ unsigned sh_ticket[kTicketRing];
+    __shared__ uint32_t sh_cC[kEmitStages][kEmitWorkers], sh_cA[kEmitStages][kEmitWorkers], sh_cB[kEmitStages][kEmitWorkers];
+    __shared__ uint32_t sh_wC[kEmitStages][kEmitWorkers], sh_wA[kEmitStages][kEmitWorkers], sh_wB[kEmitStages][kEmitWorkers];
+    __shared__ uint32_t sh_pre[kEmitStages][4];  // {C, A, B} before the tile; [3]: 1 = valid, 0 = skip the write
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int m = blockIdx.y;
-    const EmitParams e = emit[m];
-    if (!e.enabled) return;
-    if (threadIdx.x == 0) sh_ticket = atomicAdd(&tile_counter[m], 1u);
-    __syncthreads();
-    const int t = (int)sh_ticket;
-    uint4* desc = tile_desc + (int64_t)m * tiles_per_worker;
+    const uint32_t lt = (1u << lane) - 1u;
+    const unsigned kNone = 0xFFFFFFFFu;
 
-    // ---- load this thread's 16 consecutive elements
-    const T* row = g + (int64_t)m * ld;
-    const int64_t i0 = (int64_t)t * kEmitTile + (int64_t)threadIdx.x * kEmitItems;
-    uint32_t bits[kEmitItems];
-    uint32_t valid = 0;
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-        const int64_t base = i0 + j * V;
-        if (base + V <= d) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4*>(row + base));
-            if constexpr (V == 4) {
-                bits[j * 4 + 0] = q.x; bits[j * 4 + 1] = q.y; bits[j * 4 + 2] = q.z; bits[j * 4 + 3] = q.w;
-            } else {
-                bits[j * 8 + 0] = q.x & 0xFFFFu; bits[j * 8 + 1] = q.x >> 16;
-                bits[j * 8 + 2] = q.y & 0xFFFFu; bits[j * 8 + 3] = q.y >> 16;
-                bits[j * 8 + 4] = q.z & 0xFFFFu; bits[j * 8 + 5] = q.z >> 16;
-                bits[j * 8 + 6] = q.w & 0xFFFFu; bits[j * 8 + 7] = q.w >> 16;
+    if (threadIdx.x == 0) {
+        sy.tickets_ready = 0; sy.prefix_ready = 0; sy.abort = 0;
+        for (int i = 0; i < kEmitStages; ++i) sy.counted[i] = 0;
+    }
+    __syncthreads();
+
+    if (warp < kEmitWorkers) {
+        // =========================== worker warps ===========================
+        uint32_t* my_ring = sh_ring + warp * kShare;
+        auto fetch = [&](unsigned q, int k) {  // one commit per call, also for tiles that are skipped
+            if (q < total_tiles) {
+                const int mq = (int)(q % (unsigned)M);
+                if (emit[mq].enabled)
+                    emit_fetch_share<T>(g + (int64_t)mq * ld, d, (int64_t)(q / (unsigned)M),
+                                        my_ring + (k & (kEmitStages - 1)) * kEmitTile, warp, lane);
             }
-            valid |= ((1u << V) - 1u) << (j * V);
-        } else {
-#pragma unroll
-            for (int c = 0; c < V; ++c) {
-                bits[j * V + c] = 0;
-                if (base + c < d) {
-                    if constexpr (V == 4)
-                        bits[j * V + c] = reinterpret_cast<const uint32_t*>(row)[base + c];
-                    else
-                        bits[j * V + c] = reinterpret_cast<const uint16_t*>(row)[base + c];
-                    valid |= 1u << (j * V + c);
-                }
-            }
+            cp_async_commit();
+        };
+        auto ticket_of = [&](int k, unsigned* q) -> bool {
+            if (!wait_at_least(&sy.tickets_ready, (unsigned)k + 1u, &sy.abort)) return false;
+            *q = sh_ticket[k & (kTicketRing - 1)];
+            return true;
+        };
+        unsigned q_m2 = kNone, q_m1 = kNone, q_0 = kNone, q_p1 = kNone;  // tiles k-2, k-1, k, k+1
+        uint32_t fl_m2 = 0, fl_m1 = 0, ra_m2 = 0, ra_m1 = 0;              // their flags / row masks
+        bool alive = ticket_of(0, &q_0) && ticket_of(1, &q_p1);
+        if (alive) {
+            fetch(q_0, 0);
+            fetch(q_p1, 1);
         }
-    }
-
-    // ---- local counts, packed 21 bits each: D | Ea << 21 | Eb << 42
-    unsigned long long pack = 0;
+        for (int k = 0; alive && (q_0 < total_tiles || q_m2 < total_tiles || q_m1 < total_tiles); ++k) {
+            // ---- count this warp's share of tile k.
+            // flags: bit i (fp32) or bits i and 16 + i (bf16 low / high half) = word i holds a closed-range key
+            uint32_t flags = 0, rowany = 0;
+            if (q_0 < total_tiles) {
+                const int mc_ = (int)(q_0 % (unsigned)M);
+                const EmitParams ec = emit[mc_];
+                uint32_t cC = 0, cA = 0, cB = 0;
+                cp_async_wait<1>();  // the share of tile k has landed (tile k+1 may still be in flight)
+                __syncwarp();
+                if (ec.enabled) {
+                    const uint32_t* tile = my_ring + (k & (kEmitStages - 1)) * kEmitTile + lane;
+                    const uint32_t Tb = min(ec.Tb, EW::kCap), Ta = min(ec.Ta, EW::kCap);
+                    if constexpr (S == 1) {
+                        const uint32_t W = Ta - Tb;
 #pragma unroll
-    for (int i = 0; i < kEmitItems; ++i) {
-        const uint32_t key = Tr::key(bits[i]);
-        const bool ok = (valid >> i) & 1u;
-        const unsigned long long dD = (ok && key > e.Tb && key <= e.Ta) ? 1ull : 0ull;
-        const unsigned long long dA = (ok && key == e.Ta) ? 1ull : 0ull;
-        const unsigned long long dB = (ok && key == e.Tb) ? 1ull : 0ull;
-        pack += dD | (dA << 21) | (dB << 42);
-    }
-    unsigned long long inc = pack;
+                        for (int i = 0; i < kEmitRows; ++i)
+                            if (((tile[i * 32] & 0x7FFFFFFFu) - Tb) <= W) flags |= 1u << i;
+                        if (__any_sync(0xFFFFFFFFu, flags != 0u)) {  // ties are closed-range keys: look only if there are any
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= o) inc += y;
-    }
-    if (lane == 31) sh_warp[warp] = inc;
-    __syncthreads();
-    unsigned long long warp_off = 0, block_total = 0;
+                            for (int i = 0; i < kEmitRows; ++i) {
+                                const uint32_t tk = (tile[i * 32] & 0x7FFFFFFFu) - Tb;
+                                cA += (tk == W) ? 1u : 0u;
+                                cB += (tk == 0u) ? 1u : 0u;
+                            }
+                        }
+                    } else {
+                        // two 15-bit keys per word; bit 15 of each half is free, so both halves are compared at
+                        // once: (key + 0x8000 - T) has bit 15 set iff key >= T, (T + 0x8000 - key) iff key <= T
+                        const uint32_t hi = 0x80008000u;
+                        const uint32_t geB = hi - Tb * 0x10001u, geB1 = hi - (Tb + 1u) * 0x10001u;
+                        const uint32_t leA = hi + Ta * 0x10001u, leA1 = hi + (Ta ? Ta - 1u : 0u) * 0x10001u;
+                        const uint32_t keepA1 = Ta ? 0xFFFFFFFFu : 0u;  // Ta = 0: every closed key equals Ta
+                        uint32_t acc = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        const unsigned long long s = sh_warp[w];
-        if (w < warp) warp_off += s;
-        block_total += s;
-    }
-    const unsigned long long excl = inc - pack + warp_off;
-    const uint32_t aggD = (uint32_t)(block_total & 0x1FFFFFu);
-    const uint32_t aggA = (uint32_t)((block_total >> 21) & 0x1FFFFFu);
-    const uint32_t aggB = (uint32_t)((block_total >> 42) & 0x1FFFFFu);
-
-    // ---- decoupled look-back over this worker's earlier tiles (warp 0)
-    if (warp == 0) {
-        uint32_t pD = 0, pA = 0, pB = 0;
-        bool ok = true;
-        if (t > 0) {
-            if (lane == 0) put_record(&desc[t], aggD, aggA, aggB, 1u);
-            int look = t - 1;
-            unsigned spins = 0;
-            while (true) {
-                const int at = look - lane;
-                // positions before the worker's first tile count as an empty running total
-                uint4 rec = (at >= 0) ? __ldcg(&desc[at]) : make_uint4(0u, 0u, 0u, 2u);
-                while (!__all_sync(0xFFFFFFFFu, rec.w != 0u)) {
-                    if (at >= 0 && rec.w == 0u) rec = __ldcg(&desc[at]);
-                    const bool bail = (++spins > kSpinLimit) ||
-                                      (*reinterpret_cast<volatile int*>(status) == MLMC_ERR_TIMEOUT);
-                    if (__any_sync(0xFFFFFFFFu, bail)) {  // warp-uniform exit
-                        ok = false;
-                        break;
+                        for (int i = 0; i < kEmitRows; ++i) {
+                            const uint32_t k2 = tile[i * 32] & 0x7FFF7FFFu;
+                            const uint32_t f = (k2 + geB) & (leA - k2) & hi;
+                            flags |= f >> (15 - i);
+                            const uint32_t fB = f & ~(k2 + geB1);
+                            const uint32_t fA = f & ~((leA1 - k2) & keepA1);
+                            acc += (fA >> 15) + (fB >> 7);  // 5-bit counters: A at bits 0 / 16, B at bits 8 / 24
+                        }
+                        cA = (acc & 0x1Fu) + ((acc >> 16) & 0x1Fu);
+                        cB = ((acc >> 8) & 0x1Fu) + ((acc >> 24) & 0x1Fu);
+                    }
+                    rowany = __reduce_or_sync(0xFFFFFFFFu, flags);
+                    if (rowany) {
+                        const uint32_t totCA = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(flags) | (cA << 16));
+                        cB = __reduce_add_sync(0xFFFFFFFFu, cB);
+                        cC = totCA & 0xFFFFu;
+                        cA = totCA >> 16;
                     }
                 }
-                if (!ok) break;
-                const unsigned has_total = __ballot_sync(0xFFFFFFFFu, rec.w == 2u);
-                const int stop = has_total ? (__ffs(has_total) - 1) : 32;  // nearest tile with a running total
-                const bool use = lane <= stop;
-                pD += warp_sum(use ? rec.x : 0u);
-                pA += warp_sum(use ? rec.y : 0u);
-                pB += warp_sum(use ? rec.z : 0u);
-                if (has_total) break;
-                look -= 32;
-            }
-            if (!ok) {
-                set_status(status, MLMC_ERR_TIMEOUT);
-                worker_err[m] = MLMC_ERR_TIMEOUT;
-            }
-        }
-        if (lane == 0) {
-            put_record(&desc[t], pD + aggD, pA + aggA, pB + aggB, 2u);  // also after a give-up, so successors move on
-            sh_prefix[0] = pD; sh_prefix[1] = pA; sh_prefix[2] = pB; sh_prefix[3] = ok ? 1u : 0u;
-        }
-    }
-    __syncthreads();
-    const bool ok = sh_prefix[3] != 0;
-    uint32_t rD = sh_prefix[0] + (uint32_t)(excl & 0x1FFFFFu);
-    uint32_t rA = sh_prefix[1] + (uint32_t)((excl >> 21) & 0x1FFFFFu);
-    uint32_t rB = sh_prefix[2] + (uint32_t)((excl >> 42) & 0x1FFFFFu);
-
-    // ---- self-check on the worker's last tile: the band has exactly k_l - k_{l-1} entries
-    if (t == tiles_per_worker - 1 && threadIdx.x == 0 && ok) {
-        const uint32_t tD = sh_prefix[0] + aggD, tA = sh_prefix[1] + aggA, tB = sh_prefix[2] + aggB;
-        const uint32_t total = tD + min(tB, e.rb) - min(tA, e.ra);
-        if (total != e.expect) set_status(status, MLMC_ERR_INTERNAL);
-    }
-
-    // ---- write the band entries at their global positions
-    if (ok && (aggD | aggA | aggB)) {
-        uint32_t* idx_w = idx_out + (int64_t)m * capacity;
-        float* val_w = val_out + (int64_t)m * capacity;
-#pragma unroll
-        for (int i = 0; i < kEmitItems; ++i) {
-            const uint32_t key = Tr::key(bits[i]);
-            const bool okv = (valid >> i) & 1u;
-            const bool eqA = okv && key == e.Ta, eqB = okv && key == e.Tb;
-            const bool insA = okv && (key > e.Ta || (eqA && rA < e.ra));   // tie rank rA + 1 <= ra
-            const bool insB = okv && (key > e.Tb || (eqB && rB < e.rb));
-            if (insB && !insA) {
-                const uint32_t pos = rD + min(rB, e.rb) - min(rA, e.ra);
-                if ((int64_t)pos < capacity) {
-                    idx_w[pos] = (uint32_t)(i0 + i);
-                    val_w[pos] = (float)((double)Tr::value(bits[i]) * e.inv_p);
+                if (lane == 0) {
+                    const int slot = k & (kEmitStages - 1);
+                    sh_cC[slot][warp] = cC; sh_cA[slot][warp] = cA; sh_cB[slot][warp] = cB;
+                    __threadfence_block();
+                    atomicAdd(&sy.counted[slot], 1u);
                 }
             }
-            rD += (okv && key > e.Tb && key <= e.Ta) ? 1u : 0u;
-            rA += eqA ? 1u : 0u;
-            rB += eqB ? 1u : 0u;
+
+            // ---- write this warp's share of tile k-2
+            if (q_m2 < total_tiles) {
+                const int mp = (int)(q_m2 % (unsigned)M), tp = (int)(q_m2 / (unsigned)M);
+                const EmitParams ep = emit[mp];
+                const int slot = (k - 2) & (kEmitStages - 1);
+                if (!wait_at_least(&sy.prefix_ready, (unsigned)(k - 2) + 1u, &sy.abort)) {
+                    alive = false;
+                    break;
+                }
+                if (ep.enabled && ra_m2 && sh_pre[slot][3]) {
+                    const uint32_t* tile = my_ring + slot * kEmitTile + lane;
+                    const uint32_t Tb = min(ep.Tb, EW::kCap);
+                    const uint32_t W = min(ep.Ta, EW::kCap) - Tb;
+                    uint32_t rA = sh_pre[slot][1] + sh_wA[slot][warp], rB = sh_pre[slot][2] + sh_wB[slot][warp];
+                    uint32_t base = band_prefix(sh_pre[slot][0] + sh_wC[slot][warp], rA, rB, ep.ra, ep.rb);
+                    // ties in this warp's share?  (warp-uniform; ties elsewhere only move the base)
+                    const bool ties = (sh_cA[slot][warp] | sh_cB[slot][warp]) != 0u;
+                    const float inv_p = (float)ep.inv_p;
+                    uint32_t* idx_w = idx_out + (int64_t)mp * capacity;
+                    float* val_w = val_out + (int64_t)mp * capacity;
+                    const uint32_t e0 = (uint32_t)(((int64_t)tp * kEmitTile + warp * kShare + lane) * S);
+                    uint32_t rows = (ra_m2 | (ra_m2 >> 16)) & 0xFFFFu;  // rows that hold a closed-range key
+                    // rolled loops over the rows that matter: the body is long, unrolling it 16 times would not fit
+                    // the instruction cache
+#pragma unroll 1
+                    while (rows) {
+                        const int i = __ffs(rows) - 1;
+                        rows &= rows - 1u;
+                        const uint32_t w = tile[i * 32];
+                        bool em[S];
+                        uint32_t me[S];
+                        if (!ties) {
+#pragma unroll
+                            for (int s = 0; s < S; ++s) {
+                                em[s] = (fl_m2 >> (i + 16 * s)) & 1u;
+                                me[s] = __ballot_sync(0xFFFFFFFFu, em[s]);
+                            }
+                        } else {
+                            uint32_t tk[S], mA[S], mB[S], a_lt = 0, b_lt = 0;
+#pragma unroll
+                            for (int s = 0; s < S; ++s) {
+                                tk[s] = EW::key(w, s) - Tb;
+                                mA[s] = __ballot_sync(0xFFFFFFFFu, tk[s] == W);
+                                mB[s] = __ballot_sync(0xFFFFFFFFu, tk[s] == 0u);
+                                a_lt += __popc(mA[s] & lt);
+                                b_lt += __popc(mB[s] & lt);
+                            }
+#pragma unroll
+                            for (int s = 0; s < S; ++s) {
+                                // index-ordered tie ranks (0-based) of this element among the keys equal to Ta / Tb
+                                const bool inA = (tk[s] == W) && (rA + a_lt) < ep.ra;    // still inside Top-k_{l-1}
+                                const bool outB = (tk[s] == 0u) && (rB + b_lt) >= ep.rb; // already outside Top-k_l
+                                em[s] = (tk[s] <= W) && !inA && !outB;
+                                me[s] = __ballot_sync(0xFFFFFFFFu, em[s]);
+                                a_lt += (mA[s] >> lane) & 1u;
+                                b_lt += (mB[s] >> lane) & 1u;
+                            }
+#pragma unroll
+                            for (int s = 0; s < S; ++s) {
+                                rA += __popc(mA[s]);
+                                rB += __popc(mB[s]);
+                            }
+                        }
+                        uint32_t pos = base;
+#pragma unroll
+                        for (int s = 0; s < S; ++s) pos += __popc(me[s] & lt);
+#pragma unroll
+                        for (int s = 0; s < S; ++s) {
+                            if (em[s]) {
+                                if ((int64_t)pos < capacity) {
+                                    idx_w[pos] = e0 + (uint32_t)(i * 32 * S + s);
+                                    val_w[pos] = EW::value(w, s) * inv_p;
+                                }
+                                ++pos;
+                            }
+                        }
+                        base = __shfl_sync(0xFFFFFFFFu, pos, 31);  // lane 31 ends at the row's total
+                    }
+                }
+            }
+
+            // ---- start the copy of tile k+2 into the slot that tile k-2 has just left
+            unsigned q_p2 = kNone;
+            if (!ticket_of(k + 2, &q_p2)) {
+                alive = false;
+                break;
+            }
+            __syncwarp();
+            fetch(q_p2, k + 2);
+            q_m2 = q_m1; q_m1 = q_0; q_0 = q_p1; q_p1 = q_p2;
+            fl_m2 = fl_m1; fl_m1 = flags;
+            ra_m2 = ra_m1; ra_m1 = rowany;
+        }
+        cp_async_wait<0>();
+    } else {
+        // =========================== prefix warp ===========================
+        bool more = true;  // valid tickets may remain
+        auto put_ticket = [&](unsigned i, unsigned q) {
+            if (lane == 0) {
+                sh_ticket[i & (kTicketRing - 1)] = q;
+                __threadfence_block();
+                *reinterpret_cast<volatile unsigned*>(&sy.tickets_ready) = i + 1u;
+            }
+        };
+        auto take_ticket = [&]() -> unsigned {
+            unsigned q = kNone;
+            if (more && lane == 0) q = atomicAdd(tile_counter, 1u);
+            return q;
+        };
+        constexpr unsigned kAhead = 5;  // tickets kept ahead of the tile being handled (workers ask for tile k+2)
+        for (unsigned i = 0; i < kAhead; ++i) {
+            const unsigned q = __shfl_sync(0xFFFFFFFFu, take_ticket(), 0);
+            if (q >= total_tiles) more = false;
+            put_ticket(i, q);
+        }
+        // Tile j's counts are published as soon as its shares are counted; its look-back runs one tile later,
+        // while the workers count tile j+1.  By then the tiles that were counted at the same time as tile j
+        // have published their counts too, so the look-back does not wait for stragglers, and the nearest
+        // running total is about two rounds of the grid back: the window is 128 records wide.
+        constexpr int kWin = 4;  // records per lane and step
+        unsigned q_prev = kNone;
+        uint32_t aggC_p = 0, aggA_p = 0, aggB_p = 0;
+        for (unsigned j = 0;; ++j) {
+            // ask for the next ticket now, hand it out at the end of this tile: the atomic's latency stays hidden
+            const unsigned q_ahead = take_ticket();
+            const unsigned q = sh_ticket[j & (kTicketRing - 1)];
+            const bool cur_ok = q < total_tiles, prev_ok = q_prev < total_tiles;
+            if (!cur_ok && !prev_ok) break;  // tickets only grow: nothing valid follows (the tickets ahead are already out)
+            const int m = cur_ok ? (int)(q % (unsigned)M) : 0, t = cur_ok ? (int)(q / (unsigned)M) : 0;
+            const int mp = prev_ok ? (int)(q_prev % (unsigned)M) : 0, tp = prev_ok ? (int)(q_prev / (unsigned)M) : 0;
+            const EmitParams e = emit[m], ep = emit[mp];
+            const bool do_cur = cur_ok && e.enabled, do_prev = prev_ok && ep.enabled;
+            const int slot = j & (kEmitStages - 1), slot_p = (j - 1u) & (kEmitStages - 1);
+            uint4* desc = tile_desc + (int64_t)m * tiles_per_worker;
+            uint4* desc_p = tile_desc + (int64_t)mp * tiles_per_worker;
+            // first window of tile j-1's look-back: the loads fly while the workers count tile j.
+            // Lane i holds tiles look - i - 32 w, w = 0..3; positions before the worker's first tile are an empty total.
+            uint4 rec[kWin];
+#pragma unroll
+            for (int w = 0; w < kWin; ++w) {
+                const int at = tp - 1 - lane - 32 * w;
+                rec[w] = (do_prev && at >= 0) ? __ldcg(&desc_p[at]) : make_uint4(0u, 0u, 0u, 2u);
+            }
+            uint32_t aggC = 0, aggA = 0, aggB = 0;
+            if (cur_ok) {
+                if (!wait_at_least(&sy.counted[slot], (j / kEmitStages + 1u) * kEmitWorkers, &sy.abort)) break;
+                if (do_cur) {
+                    const uint32_t xC = (lane < kEmitWorkers) ? sh_cC[slot][lane] : 0u, xA = (lane < kEmitWorkers) ? sh_cA[slot][lane] : 0u,
+                                   xB = (lane < kEmitWorkers) ? sh_cB[slot][lane] : 0u;
+                    uint32_t iC = xC, iA = xA, iB = xB;
+#pragma unroll
+                    for (int o = 1; o < kEmitWorkers; o <<= 1) {
+                        const uint32_t yC = __shfl_up_sync(0xFFFFFFFFu, iC, o), yA = __shfl_up_sync(0xFFFFFFFFu, iA, o),
+                                       yB = __shfl_up_sync(0xFFFFFFFFu, iB, o);
+                        if (lane >= o) { iC += yC; iA += yA; iB += yB; }
+                    }
+                    if (lane < kEmitWorkers) {
+                        sh_wC[slot][lane] = iC - xC;
+                        sh_wA[slot][lane] = iA - xA;
+                        sh_wB[slot][lane] = iB - xB;
+                    }
+                    aggC = __shfl_sync(0xFFFFFFFFu, iC, kEmitWorkers - 1);
+                    aggA = __shfl_sync(0xFFFFFFFFu, iA, kEmitWorkers - 1);
+                    aggB = __shfl_sync(0xFFFFFFFFu, iB, kEmitWorkers - 1);
+                    // a worker's first tile has nothing before it: its counts are already running totals
+                    if (lane == 0) put_record(&desc[t], aggC, aggA, aggB, t == 0 ? 2u : 1u);
+                }
+            }
+            if (prev_ok) {
+                uint32_t pC = 0, pA = 0, pB = 0;
+                bool ok = true;
+                if (do_prev && tp > 0) {
+                    int look = tp - 1;
+                    unsigned spins = 0;
+                    while (true) {
+                        // nearest tile with a running total: everything nearer contributes its own counts,
+                        // everything farther is not needed (and not waited for)
+                        unsigned tot[kWin];
+                        int stop[kWin];
+                        while (true) {
+                            bool found = false, pending = false;
+#pragma unroll
+                            for (int w = 0; w < kWin; ++w) {
+                                tot[w] = __ballot_sync(0xFFFFFFFFu, rec[w].w == 2u);
+                                stop[w] = found ? -1 : (tot[w] ? (__ffs(tot[w]) - 1) : 32);
+                                found |= tot[w] != 0u;
+                                pending |= (lane <= stop[w]) && rec[w].w == 0u;
+                            }
+                            if (!__any_sync(0xFFFFFFFFu, pending)) break;
+#pragma unroll
+                            for (int w = 0; w < kWin; ++w) {
+                                const int at = look - lane - 32 * w;
+                                if (at >= 0 && rec[w].w == 0u) rec[w] = __ldcg(&desc_p[at]);
+                            }
+                            const bool bail = (++spins > kLookbackSpinLimit) || *reinterpret_cast<volatile int*>(&sy.abort) ||
+                                              (*reinterpret_cast<volatile int*>(status) == MLMC_ERR_TIMEOUT);
+                            if (__any_sync(0xFFFFFFFFu, bail)) {  // warp-uniform exit
+                                ok = false;
+                                break;
+                            }
+                        }
+                        if (!ok) break;
+                        uint32_t sC = 0, sA = 0, sB = 0;
+                        unsigned any_tot = 0;
+#pragma unroll
+                        for (int w = 0; w < kWin; ++w) {
+                            const bool use = lane <= stop[w];
+                            sC += use ? rec[w].x : 0u;
+                            sA += use ? rec[w].y : 0u;
+                            sB += use ? rec[w].z : 0u;
+                            any_tot |= tot[w];
+                        }
+                        pC += __reduce_add_sync(0xFFFFFFFFu, sC);
+                        pA += __reduce_add_sync(0xFFFFFFFFu, sA);
+                        pB += __reduce_add_sync(0xFFFFFFFFu, sB);
+                        if (any_tot) break;
+                        look -= 32 * kWin;
+#pragma unroll
+                        for (int w = 0; w < kWin; ++w) {
+                            const int at = look - lane - 32 * w;
+                            rec[w] = (at >= 0) ? __ldcg(&desc_p[at]) : make_uint4(0u, 0u, 0u, 2u);
+                        }
+                    }
+                    if (lane == 0) put_record(&desc_p[tp], pC + aggC_p, pA + aggA_p, pB + aggB_p, 2u);  // also after a give-up
+                    if (!ok) {
+                        set_status(status, MLMC_ERR_TIMEOUT);
+                        worker_err[mp] = MLMC_ERR_TIMEOUT;
+                    }
+                }
+                // self-check on the worker's last tile: the band has exactly k_l - k_{l-1} entries
+                if (lane == 0 && do_prev && ok && tp == tiles_per_worker - 1 &&
+                    band_prefix(pC + aggC_p, pA + aggA_p, pB + aggB_p, ep.ra, ep.rb) != ep.expect)
+                    set_status(status, MLMC_ERR_INTERNAL);
+                if (lane == 0) {
+                    sh_pre[slot_p][0] = pC; sh_pre[slot_p][1] = pA; sh_pre[slot_p][2] = pB;
+                    sh_pre[slot_p][3] = (do_prev && ok) ? 1u : 0u;
+                    __threadfence_block();
+                    *reinterpret_cast<volatile unsigned*>(&sy.prefix_ready) = j;  // tiles [0, j) have their prefix
+                }
+            }
+            const unsigned qa = __shfl_sync(0xFFFFFFFFu, q_ahead, 0);
+            if (qa >= total_tiles) more = false;
+            put_ticket(j + kAhead, qa);
+            q_prev = q;
+            aggC_p = aggC; aggA_p = aggA; aggB_p = aggB;
         }
     }
+    if (*reinterpret_cast<volatile int*>(&sy.abort)) set_status(status, MLMC_ERR_TIMEOUT);
 }
 
 // offsets[m][t] = first message entry of worker m whose index is >= t * kAggTile  (t = 0..ntiles)
@@ -247,20 +546,35 @@ aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict_
 
 }  // namespace
 
+int configure_emit_kernels() {
+    const int smem = kEmitStages * kEmitTile * (int)sizeof(uint32_t);
+    if (cudaFuncSetAttribute(emit_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    if (cudaFuncSetAttribute(emit_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    return MLMC_OK;
+}
+
 void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const mlmc_topk_msgs& out,
                  cudaStream_t s) {
-    const int tpw = (int)((d + kEmitTile - 1) / kEmitTile);
-    cudaMemsetAsync(ws.tile_desc, 0, (size_t)tpw * M * sizeof(uint4), s);
-    cudaMemsetAsync(ws.tile_counter, 0, sizeof(unsigned) * M, s);
+    const int per_word = (dtype == MLMC_BF16) ? 2 : 1;
+    const int64_t words = (d + per_word - 1) / per_word;
+    const int tpw = (int)((words + kEmitTile - 1) / kEmitTile);
+    const unsigned total = (unsigned)tpw * (unsigned)M;
+    cudaMemsetAsync(ws.tile_desc, 0, (size_t)total * sizeof(uint4), s);
+    cudaMemsetAsync(ws.tile_counter, 0, sizeof(unsigned), s);
+    unsigned grid = (unsigned)(ws.sm_count * kEmitBlocksPerSM);  // persistent blocks
+    if (grid > total) grid = total;
+    const size_t smem = (size_t)kEmitStages * kEmitTile * sizeof(uint32_t);
     LaunchScope t(ws, K_EMIT, s);
     if (dtype == MLMC_BF16)
-        emit_kernel<bf16_t><<<dim3(tpw, M), kEmitThreads, 0, s>>>(static_cast<const bf16_t*>(g), d, ld, tpw, ws.emit,
-                                                                 ws.tile_desc, ws.tile_counter, out.idx, out.val,
-                                                                 out.capacity, ws.status, ws.worker_err);
+        emit_kernel<bf16_t><<<grid, kEmitThreads, smem, s>>>(static_cast<const bf16_t*>(g), d, ld, tpw, total, M, ws.emit,
+                                                           ws.tile_desc, ws.tile_counter, out.idx, out.val, out.capacity,
+                                                           ws.status, ws.worker_err);
     else
-        emit_kernel<float><<<dim3(tpw, M), kEmitThreads, 0, s>>>(static_cast<const float*>(g), d, ld, tpw, ws.emit,
-                                                                ws.tile_desc, ws.tile_counter, out.idx, out.val,
-                                                                out.capacity, ws.status, ws.worker_err);
+        emit_kernel<float><<<grid, kEmitThreads, smem, s>>>(static_cast<const float*>(g), d, ld, tpw, total, M, ws.emit,
+                                                          ws.tile_desc, ws.tile_counter, out.idx, out.val, out.capacity,
+                                                          ws.status, ws.worker_err);
 }
 
 void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int64_t d, float* out, cudaStream_t s) {
