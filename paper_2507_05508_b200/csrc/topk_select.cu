@@ -88,14 +88,30 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
     int64_t v0, v1;
     block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
     bool bad = false;
-#pragma unroll 4
-    for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
-        for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) {
-            const uint32_t key = Tr::key(bits);
-            bad |= (key >= Tr::kInfKey);
-            atomicAdd(&sh_hist[key >> Tr::kShift1], 1u);
-        });
+    auto count_key = [&](uint32_t bits) {
+        const uint32_t key = Tr::key(bits);
+        bad |= (key >= Tr::kInfKey);
+        atomicAdd(&sh_hist[key >> Tr::kShift1], 1u);
+    };
+    // four 16-byte loads per thread are issued before any of them is used: 64 KB in flight per SM
+    constexpr int kBatch = 4;
+    const int64_t full_end = min(v1, d / Tr::kVec);  // vectors that lie wholly inside the row
+    int64_t v = v0 + threadIdx.x;
+    for (; v + (int64_t)(kBatch - 1) * blockDim.x < full_end; v += (int64_t)kBatch * blockDim.x) {
+        uint4 q[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v + (int64_t)j * blockDim.x);
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            if constexpr (Tr::kVec == 4) {
+                count_key(q[j].x); count_key(q[j].y); count_key(q[j].z); count_key(q[j].w);
+            } else {
+                count_key(q[j].x & 0xFFFFu); count_key(q[j].x >> 16); count_key(q[j].y & 0xFFFFu); count_key(q[j].y >> 16);
+                count_key(q[j].z & 0xFFFFu); count_key(q[j].z >> 16); count_key(q[j].w & 0xFFFFu); count_key(q[j].w >> 16);
+            }
+        }
     }
+    for (; v < v1; v += blockDim.x) for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) { count_key(bits); });
     if (bad) {
         worker_err[m] = MLMC_ERR_NONFINITE;
         set_status(status, MLMC_ERR_NONFINITE);
@@ -238,25 +254,38 @@ constexpr int kS2Vecs = 4;                                   // 16-byte vectors 
 constexpr int kS2Round = kS2Threads * kS2Vecs * 4;            // elements per round
 constexpr int kStage = 2 * kS2Round;                          // staged candidate keys per block
 
-template <bool SUMS>
-__global__ void __launch_bounds__(kS2Threads)
-sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table1, int L,
-                       double* __restrict__ sum_partial, int sum_ctas, uint32_t* __restrict__ cand_keys,
-                       int64_t cand_cap, uint32_t* cand_count, int* cand_overflow, const int* worker_err) {
+// table: bin -> code.  code < 64: the bin lies wholly inside open interval `code` (between two thresholds);
+// code >= 64: the bin may hold a threshold, its keys are compacted into the candidate buffer.
+// SUMS: per-interval energy of the threshold-free bins (adaptive p).  COUNTS: per-interval element counts
+// (needed when the table comes from a sample and has to be verified).  gate (optional): only workers with
+// gate[m] != 0 are processed.  Loads are double-buffered in registers: the next round's four 16-byte
+// vectors are in flight while the current round is processed.
+template <bool SUMS, bool COUNTS>
+__global__ void __launch_bounds__(kS2Threads, 2)
+sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table, int L,
+                       double* __restrict__ sum_partial, uint32_t* __restrict__ region_partial, int sum_ctas,
+                       uint32_t* __restrict__ cand_keys, int64_t cand_cap, uint32_t* cand_count, int* cand_overflow,
+                       const int* worker_err, const int* __restrict__ gate) {
     extern __shared__ __align__(16) uint8_t sh_raw[];
     uint8_t* sh_table = sh_raw;                                                   // [32768]
     uint32_t* sh_stage = reinterpret_cast<uint32_t*>(sh_raw + kBins1);            // [kStage]
-    double* sh_acc = reinterpret_cast<double*>(sh_raw + kBins1 + kStage * 4);     // [L][kS2Threads]
+    double* sh_acc = reinterpret_cast<double*>(sh_raw + kBins1 + kStage * 4);     // [L][kS2Threads]  (SUMS)
+    uint32_t* sh_cnt = reinterpret_cast<uint32_t*>(sh_raw + kBins1 + kStage * 4 +
+                                                   (SUMS ? (size_t)L * kS2Threads * sizeof(double) : 0));  // [L][kS2Threads]
     __shared__ uint32_t sh_n;
     __shared__ uint32_t sh_base;
+    __shared__ uint32_t sh_tot[kMaxLevels];
     const int m = blockIdx.y;
-    if (worker_err[m]) return;
+    if (worker_err[m] || (gate && !gate[m])) return;
     {
-        const uint4* src = reinterpret_cast<const uint4*>(table1 + (int64_t)m * kBins1);
+        const uint4* src = reinterpret_cast<const uint4*>(table + (int64_t)m * kBins1);
         uint4* dst = reinterpret_cast<uint4*>(sh_table);
         for (int i = threadIdx.x; i < kBins1 / 16; i += kS2Threads) dst[i] = src[i];
         if (SUMS)
             for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_acc[i] = 0.0;
+        if (COUNTS)
+            for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_cnt[i] = 0u;
+        if (threadIdx.x < kMaxLevels) sh_tot[threadIdx.x] = 0u;
         if (threadIdx.x == 0) sh_n = 0;
     }
     __syncthreads();
@@ -264,6 +293,7 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
     uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
     int64_t v0, v1;
     block_vector_range(d, 4, blockIdx.x, gridDim.x, &v0, &v1);
+    const int64_t full_end = min(v1, d / 4);  // vectors wholly inside the row
 
     auto flush = [&]() {  // called by all threads
         const uint32_t n = sh_n;
@@ -281,44 +311,45 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
         if (threadIdx.x == 0) sh_n = 0;
         __syncthreads();
     };
-
-    for (int64_t vb = v0; vb < v1; vb += kS2Threads * kS2Vecs) {
-        uint4 q[kS2Vecs];
-        bool full[kS2Vecs];
-#pragma unroll
-        for (int j = 0; j < kS2Vecs; ++j) {
-            const int64_t v = vb + j * kS2Threads + threadIdx.x;
-            full[j] = (v < v1) && (v * 4 + 4 <= d);
-            if (full[j]) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v);
-        }
-#pragma unroll
-        for (int j = 0; j < kS2Vecs; ++j) {
-            const int64_t v = vb + j * kS2Threads + threadIdx.x;
-            uint32_t bits[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
-            int cnt = full[j] ? 4 : 0;
-            if (!full[j] && v < v1) {  // ragged tail of the row
-                cnt = (int)(d - v * 4);
-                for (int c = 0; c < cnt; ++c) bits[c] = reinterpret_cast<const uint32_t*>(row)[v * 4 + c];
+    auto take = [&](uint32_t bits) {
+        const uint32_t key = bits & 0x7FFFFFFFu;
+        const uint32_t code = sh_table[key >> 16];
+        if (code < 64u) {
+            if (SUMS) {
+                const double x = (double)__uint_as_float(key);
+                double* a = &sh_acc[code * kS2Threads + threadIdx.x];
+                *a = fma(x, x, *a);
             }
+            if (COUNTS) sh_cnt[code * kS2Threads + threadIdx.x] += 1u;
+        } else {
+            sh_stage[atomicAdd(&sh_n, 1u)] = key;
+        }
+    };
+    auto load_round = [&](int64_t vb, uint4 (&q)[kS2Vecs]) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (c < cnt) {
-                    const uint32_t key = bits[c] & 0x7FFFFFFFu;
-                    const uint32_t code = sh_table[key >> 16];
-                    if (code < 64u) {
-                        if (SUMS) {
-                            const double x = (double)__uint_as_float(key);
-                            double* a = &sh_acc[code * kS2Threads + threadIdx.x];
-                            *a = fma(x, x, *a);
-                        }
-                    } else {
-                        sh_stage[atomicAdd(&sh_n, 1u)] = key;
-                    }
-                }
+        for (int j = 0; j < kS2Vecs; ++j) {
+            const int64_t v = vb + j * kS2Threads + threadIdx.x;
+            if (v < full_end) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v);
+        }
+    };
+
+    uint4 cur[kS2Vecs], nxt[kS2Vecs];
+    load_round(v0, cur);
+    for (int64_t vb = v0; vb < v1; vb += kS2Threads * kS2Vecs) {
+        load_round(vb + kS2Threads * kS2Vecs, nxt);
+#pragma unroll
+        for (int j = 0; j < kS2Vecs; ++j) {
+            const int64_t v = vb + j * kS2Threads + threadIdx.x;
+            if (v < full_end) {
+                take(cur[j].x); take(cur[j].y); take(cur[j].z); take(cur[j].w);
+            } else if (v < v1) {  // ragged tail of the row
+                for (int64_t i = v * 4; i < d; ++i) take(reinterpret_cast<const uint32_t*>(row)[i]);
             }
         }
         __syncthreads();
         if (sh_n > (uint32_t)(kStage - kS2Round)) flush();  // uniform: sh_n is read after the barrier
+#pragma unroll
+        for (int j = 0; j < kS2Vecs; ++j) cur[j] = nxt[j];
     }
     flush();
     if (SUMS) {
@@ -330,6 +361,14 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
             }
             if (threadIdx.x == 0) sum_partial[((int64_t)m * sum_ctas + blockIdx.x) * kMaxLevels + l] = a[0];
         }
+    }
+    if (COUNTS) {
+        for (int l = 0; l < L; ++l) {
+            const uint32_t c = sh_cnt[l * kS2Threads + threadIdx.x];
+            if (c) atomicAdd(&sh_tot[l], c);
+        }
+        __syncthreads();
+        if (threadIdx.x < L) region_partial[((int64_t)m * sum_ctas + blockIdx.x) * kMaxLevels + threadIdx.x] = sh_tot[threadIdx.x];
     }
 }
 
@@ -822,24 +861,29 @@ static int cand_blocks(const Workspace& ws, int M) {
     return nb < 1 ? 1 : nb;
 }
 
+static size_t s2_smem(int L, bool sums, bool counts) {
+    return kBins1 + (size_t)kStage * 4 + (sums ? (size_t)L * kS2Threads * sizeof(double) : 0) +
+           (counts ? (size_t)L * kS2Threads * sizeof(uint32_t) : 0);
+}
+
 // Sweep 2: energies of the threshold-free bins (adaptive only) and the candidate keys of the boundary bins.
 void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,
                             cudaStream_t s) {
     cudaMemsetAsync(ws.cand_count, 0, sizeof(uint32_t) * M, s);
     cudaMemsetAsync(ws.cand_overflow, 0, sizeof(int) * M, s);
-    int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, 4);
+    int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, 2);
     if (nb > ws.sum_ctas) nb = ws.sum_ctas;
     ws.cur_sum_ctas = nb;
-    const size_t smem = kBins1 + (size_t)kStage * 4 + (sums ? (size_t)L * kS2Threads * sizeof(double) : 0);
+    const size_t smem = s2_smem(L, sums, false);
     LaunchScope t(ws, K_SUMS_CAND, s);
     if (sums)
-        sums_candidates_kernel<true><<<dim3(nb, M), kS2Threads, smem, s>>>(
-            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys, ws.cand_cap,
-            ws.cand_count, ws.cand_overflow, ws.worker_err);
+        sums_candidates_kernel<true, false><<<dim3(nb, M), kS2Threads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, nullptr, ws.sum_ctas, ws.cand_keys,
+            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr);
     else
-        sums_candidates_kernel<false><<<dim3(nb, M), kS2Threads, smem, s>>>(
-            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys, ws.cand_cap,
-            ws.cand_count, ws.cand_overflow, ws.worker_err);
+        sums_candidates_kernel<false, false><<<dim3(nb, M), kS2Threads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, nullptr, ws.sum_ctas, ws.cand_keys,
+            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr);
 }
 
 // Digit pass 2 or 3: over the candidate keys, and (early exit unless the buffer overflowed) over the full row.
@@ -941,10 +985,10 @@ int configure_select_kernels() {
     e = cudaFuncSetAttribute(norm_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxLevels * kSweepThreads * sizeof(double)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
-    const int smem_s2 = kBins1 + kStage * 4 + kMaxLevels * kS2Threads * (int)sizeof(double);
-    e = cudaFuncSetAttribute(sums_candidates_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
+    const int smem_s2 = (int)s2_smem(kMaxLevels, true, false);  // 160 KB; with counts as well L is limited (see launcher)
+    e = cudaFuncSetAttribute(sums_candidates_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
-    e = cudaFuncSetAttribute(sums_candidates_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
+    e = cudaFuncSetAttribute(sums_candidates_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     e = cudaFuncSetAttribute(cand_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxLevels * 4 * kCandSumThreads * sizeof(unsigned long long)));
