@@ -28,7 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         cmd = [nvcc] + NVCC_FLAGS + [os.path.join(CSRC, f) for f in SOURCES] + ["-o", LIB]
         res = subprocess.run(cmd, capture_output=True, text=True)
-        if verbose or res.returncode != 0:
+        if verbose or res.returncode != 0:  # noqa
             print(res.stdout)
             print(res.stderr)
         if res.returncode != 0:

@@ -121,7 +121,9 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     if (!guard.ok) return MLMC_ERR_CUDA;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MLMC_ERR_CUDA;
-    if (configure_select_kernels() != MLMC_OK || configure_emit_kernels() != MLMC_OK) return MLMC_ERR_CUDA;
+    if (configure_select_kernels() != MLMC_OK || configure_emit_kernels() != MLMC_OK ||
+        configure_bit_kernels() != MLMC_OK)
+        return MLMC_ERR_CUDA;
 
     mlmc_ctx* ctx = new (std::nothrow) mlmc_ctx();
     if (!ctx) return MLMC_ERR_NOMEM;

@@ -42,8 +42,28 @@ absmax_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* gmax_bit
     int64_t v0, v1;
     block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
     uint32_t mx = 0;
-#pragma unroll 4
-    for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x)
+    // four 16-byte loads per thread are in flight before any is used
+    constexpr int kBatch = 4;
+    const int64_t full_end = min(v1, d / Tr::kVec);  // vectors wholly inside the row
+    int64_t v = v0 + threadIdx.x;
+    for (; v + (int64_t)(kBatch - 1) * blockDim.x < full_end; v += (int64_t)kBatch * blockDim.x) {
+        uint4 q[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v + (int64_t)j * blockDim.x);
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            if constexpr (Tr::kVec == 4) {
+                mx = max(max(mx, q[j].x & 0x7FFFFFFFu), max(q[j].y & 0x7FFFFFFFu, max(q[j].z & 0x7FFFFFFFu, q[j].w & 0x7FFFFFFFu)));
+            } else {
+                // both halves at once: the low halves after masking, the high halves shifted down
+                const uint32_t a = max(max(q[j].x & 0x7FFFu, q[j].y & 0x7FFFu), max(q[j].z & 0x7FFFu, q[j].w & 0x7FFFu));
+                const uint32_t b = max(max((q[j].x >> 16) & 0x7FFFu, (q[j].y >> 16) & 0x7FFFu),
+                                       max((q[j].z >> 16) & 0x7FFFu, (q[j].w >> 16) & 0x7FFFu));
+                mx = max(mx, max(a, b));
+            }
+        }
+    }
+    for (; v < v1; v += blockDim.x)
         for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) { mx = max(mx, Tr::key(bits)); });
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
@@ -73,26 +93,46 @@ bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t*
     const float two_b = (float)(1u << sc.B);
     const uint32_t qmax = (1u << sc.B) - 1u;
     unsigned long long acc[LMAX];
+    int sh[LMAX];
+    uint32_t mk[LMAX];
 #pragma unroll
-    for (int l = 0; l < LMAX; ++l) acc[l] = 0;
+    for (int l = 0; l < LMAX; ++l) {  // the schedule in registers; levels past L get an empty mask and add nothing
+        acc[l] = 0;
+        sh[l] = (l < sc.L) ? sc.shift[l] : 0;
+        mk[l] = (l < sc.L) ? sc.mask[l] : 0u;
+    }
     if (gmax > 0.0f) {
         const T* row = g + (int64_t)m * ld;
         int64_t v0, v1;
         block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
-#pragma unroll 2
-        for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
-            for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) {
-                const float mag = fabsf(Tr::value(bits));
-                const uint32_t q = fixed_point_code(mag, gmax, two_b, qmax);
+        auto take = [&](uint32_t bits) {
+            const float mag = fabsf(Tr::value(bits));
+            const uint32_t q = fixed_point_code(mag, gmax, two_b, qmax);
 #pragma unroll
-                for (int l = 0; l < LMAX; ++l) {
-                    if (l < sc.L) {
-                        const uint32_t f = (q >> sc.shift[l]) & sc.mask[l];
-                        acc[l] += (unsigned long long)f * f;
-                    }
+            for (int l = 0; l < LMAX; ++l) {
+                const uint32_t f = (q >> sh[l]) & mk[l];
+                acc[l] += (unsigned long long)f * f;
+            }
+        };
+        // two 16-byte loads per thread are in flight before either is used
+        constexpr int kBatch = 2;
+        const int64_t full_end = min(v1, d / Tr::kVec);  // vectors wholly inside the row
+        int64_t v = v0 + threadIdx.x;
+        for (; v + (int64_t)(kBatch - 1) * blockDim.x < full_end; v += (int64_t)kBatch * blockDim.x) {
+            uint4 qv[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) qv[j] = __ldg(reinterpret_cast<const uint4*>(row) + v + (int64_t)j * blockDim.x);
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                if constexpr (Tr::kVec == 4) {
+                    take(qv[j].x); take(qv[j].y); take(qv[j].z); take(qv[j].w);
+                } else {
+                    take(qv[j].x & 0xFFFFu); take(qv[j].x >> 16); take(qv[j].y & 0xFFFFu); take(qv[j].y >> 16);
+                    take(qv[j].z & 0xFFFFu); take(qv[j].z >> 16); take(qv[j].w & 0xFFFFu); take(qv[j].w >> 16);
                 }
-            });
+            }
         }
+        for (; v < v1; v += blockDim.x) for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) { take(bits); });
     }
 #pragma unroll
     for (int l = 0; l < LMAX; ++l) {
@@ -178,17 +218,22 @@ __global__ void bit_probs_draw_kernel(BitSchedule sc, const uint32_t* gmax_bits,
     bit_level[m] = level;
 }
 
-// ---- pack: every warp turns 1024 consecutive entries into 32 words of each plane
+// ---- pack: every warp turns 1024 consecutive entries into 32 words of each plane.
+// The entries of a group are staged in a two-slot shared-memory ring private to the warp: the next group's
+// copy (cp.async) is in flight while the current group is coded and packed.
 template <typename T>
-__global__ void __launch_bounds__(kBitThreads)
+__global__ void __launch_bounds__(kBitThreads, 2)
 bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* __restrict__ gmax_bits,
                 BitSchedule sc, const int32_t* __restrict__ bit_level, uint32_t* __restrict__ planes, int w_max,
                 int64_t words) {
     using Tr = ElemTraits<T>;
+    constexpr int kGroup = 1024;
+    constexpr int kGroupBytes = kGroup * (int)sizeof(T);
+    extern __shared__ __align__(16) uint8_t sh_pack[];  // [warps][2][kGroupBytes]
     const int m = blockIdx.y;
     const int level = bit_level[m];
     if (level < 0) return;
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int warps_per_block = kBitThreads / 32;
     const int64_t ngroups = (words + 31) / 32;  // groups of 32 words = 1024 entries
     const float gmax = __uint_as_float(gmax_bits[m]);
@@ -199,25 +244,45 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
     const int w = sc.width[level];
     const T* row = g + (int64_t)m * ld;
     uint32_t* out = planes + (int64_t)m * (1 + w_max) * words;
-    for (int64_t grp = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); grp < ngroups;
-         grp += (int64_t)gridDim.x * warps_per_block) {
-        const int64_t e0 = grp * 1024;
+    uint8_t* ring = sh_pack + warp * 2 * kGroupBytes;
+    auto fetch = [&](int64_t grp, int stage) {  // one commit per call
+        if (grp < ngroups) {
+            const int64_t e0 = grp * kGroup;
+            uint8_t* dst = ring + stage * kGroupBytes;
+            if (e0 + kGroup <= d) {
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(row + e0);
+#pragma unroll
+                for (int c = lane; c < kGroupBytes / 16; c += 32) cp_async_16(dst + c * 16, src + c * 16);
+            } else {  // ragged last group: entries past d read as +0
+                for (int i = lane; i < kGroup; i += 32) {
+                    if constexpr (Tr::kVec == 4)
+                        reinterpret_cast<uint32_t*>(dst)[i] = (e0 + i < d) ? reinterpret_cast<const uint32_t*>(row)[e0 + i] : 0u;
+                    else
+                        reinterpret_cast<uint16_t*>(dst)[i] = (e0 + i < d) ? reinterpret_cast<const uint16_t*>(row)[e0 + i] : (uint16_t)0;
+                }
+            }
+        }
+        cp_async_commit();
+    };
+    const int64_t stride = (int64_t)gridDim.x * warps_per_block;
+    int64_t grp = (int64_t)blockIdx.x * warps_per_block + warp;
+    fetch(grp, 0);
+    for (int it = 0; grp < ngroups; grp += stride, ++it) {
+        fetch(grp + stride, (it + 1) & 1);
+        cp_async_wait<1>();  // this group has landed (the next one may still be in flight)
+        __syncwarp();
+        const uint8_t* buf = ring + (it & 1) * kGroupBytes;
         uint32_t code[32];  // bit 31 = sign, low bits = field
 #pragma unroll
         for (int s = 0; s < 32; ++s) {
-            const int64_t i = e0 + s * 32 + lane;
-            uint32_t c = 0;
-            if (i < d) {
-                uint32_t bits;
-                if constexpr (Tr::kVec == 4)
-                    bits = __ldg(reinterpret_cast<const uint32_t*>(row) + i);
-                else
-                    bits = __ldg(reinterpret_cast<const uint16_t*>(row) + i);
-                const float x = Tr::value(bits);
-                const uint32_t q = (gmax > 0.0f) ? fixed_point_code(fabsf(x), gmax, two_b, qmax) : 0u;
-                c = ((q >> shift) & mask) | (__float_as_uint(x) & 0x80000000u);
-            }
-            code[s] = c;
+            uint32_t bits;
+            if constexpr (Tr::kVec == 4)
+                bits = reinterpret_cast<const uint32_t*>(buf)[s * 32 + lane];
+            else
+                bits = reinterpret_cast<const uint16_t*>(buf)[s * 32 + lane];
+            const float x = Tr::value(bits);
+            const uint32_t q = (gmax > 0.0f) ? fixed_point_code(fabsf(x), gmax, two_b, qmax) : 0u;
+            code[s] = ((q >> shift) & mask) | (__float_as_uint(x) & 0x80000000u);
         }
         const int64_t word = grp * 32 + lane;
         for (int j = 0; j <= w; ++j) {
@@ -230,7 +295,9 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
             }
             if (word < words) out[(int64_t)j * words + word] = mine;
         }
+        __syncwarp();  // everyone is done with this slot before the copy after next lands in it
     }
+    cp_async_wait<0>();
 }
 
 // ---- server average of bit-plane messages: thread = one word (32 entries), staged through shared memory
@@ -307,6 +374,13 @@ int bit_blocks(const Workspace& ws, int64_t d, int vec, int M, int waves) {
 
 }  // namespace
 
+int configure_bit_kernels() {
+    if (cudaFuncSetAttribute(bit_pack_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (kBitThreads / 32) * 2 * 1024 * 4) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    return MLMC_OK;
+}
+
 void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
     cudaMemsetAsync(ws.gmax_bits, 0, (size_t)M * sizeof(uint32_t), s);
     LaunchScope t(ws, K_ABSMAX, s);
@@ -366,15 +440,15 @@ void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, 
     const int64_t words = (d + 31) / 32;
     const int64_t ngroups = (words + 31) / 32;
     int64_t nb = (ngroups + (kBitThreads / 32) - 1) / (kBitThreads / 32);
-    const int64_t cap = ((int64_t)ws.sm_count * 16 + M - 1) / M;
+    const int64_t cap = ((int64_t)ws.sm_count * 2 + M - 1) / M;  // persistent: two resident blocks per SM
     if (nb > cap) nb = cap;
     if (nb < 1) nb = 1;
     LaunchScope t(ws, K_BIT_PACK, s);
     if (dtype == MLMC_BF16)
-        bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, 0, s>>>(
+        bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * 2 * 1024 * 2, s>>>(
             static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
     else
-        bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, 0, s>>>(
+        bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * 2 * 1024 * 4, s>>>(
             static_cast<const float*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
 }
 

@@ -187,6 +187,15 @@ __device__ __forceinline__ void for_each_in_vector(const T* row, int64_t v, int6
     }
 }
 
+// 16-byte asynchronous copy from global to shared memory (cp.async), grouped by commit / wait.
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+    const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sa), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
 // Contiguous range of 16-byte vectors handled by block `bx` of `nb` blocks over a row of d elements.
 __device__ __forceinline__ void block_vector_range(int64_t d, int vec, int bx, int nb, int64_t* v0, int64_t* v1) {
     const int64_t nvec = (d + vec - 1) / vec;
@@ -240,6 +249,7 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
                  cudaStream_t s);
 void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int64_t d, float* out, cudaStream_t s);
 // bitwise.cu
+int configure_bit_kernels();
 void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s);
 void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
                       cudaStream_t s);

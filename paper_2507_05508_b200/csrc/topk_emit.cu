@@ -28,14 +28,6 @@ __device__ __forceinline__ void put_record(uint4* rec, uint32_t C, uint32_t A, u
     __stcg(rec, make_uint4(C, A, B, state));
 }
 
-__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
-    const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sa), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
 // How a 32-bit word of the gradient row maps to elements: one fp32 element, or two bf16 elements
 // (low half first).  A word past the end of the row reads as kPad, whose keys lie above every
 // threshold the kernel uses (thresholds are clamped to kCap, the key of +Inf), so padded elements
