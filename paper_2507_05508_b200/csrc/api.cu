@@ -145,6 +145,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     // candidate keys: a quarter of the row (boundary bins normally hold a few percent of it); small rows fit whole
     ws.cand_cap = d_max / 4 > (int64_t(1) << 20) ? d_max / 4 : (d_max < (int64_t(1) << 20) ? d_max : (int64_t(1) << 20));
     ws.stat_ctas = ws.sm_count * 4;
+    ws.cur_stat_ctas = 0;
     const int64_t emit_tiles = (d_max + kEmitTile - 1) / kEmitTile;
     const int64_t agg_tiles = (d_max + kAggTile - 1) / kAggTile;
     ws.max_tiles = emit_tiles * M_max;

@@ -164,21 +164,24 @@ __device__ int draw_level_bits(const double* p, int L, double u) {
     return 0;
 }
 
-// ---- probabilities, draw and message header of every worker (one thread per worker)
+// ---- probabilities, draw and message header of every worker (one warp per worker)
 __global__ void bit_probs_draw_kernel(BitSchedule sc, const uint32_t* gmax_bits, const unsigned long long* S_partial,
                                       int n_partials, int stat_ctas, const double* p_fixed, int adaptive,
                                       int need_delta, uint64_t seed, uint64_t step, int M, double* p_all,
                                       double* delta_all, double* u_dev, int32_t* bit_level, float* out_gmax,
                                       int32_t* out_level, double* out_p_sel, int w_max, int want_msg, int* status,
                                       int* worker_err) {
-    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    const int m = blockIdx.x;
+    const int lane = threadIdx.x;
     if (m >= M) return;
     if (worker_err[m]) {
-        bit_level[m] = -1;
-        if (want_msg) {
-            out_level[m] = -1;
-            out_p_sel[m] = 0.0;
-            out_gmax[m] = 0.0f;
+        if (lane == 0) {
+            bit_level[m] = -1;
+            if (want_msg) {
+                out_level[m] = -1;
+                out_p_sel[m] = 0.0;
+                out_gmax[m] = 0.0f;
+            }
         }
         return;
     }
@@ -186,14 +189,25 @@ __global__ void bit_probs_draw_kernel(BitSchedule sc, const uint32_t* gmax_bits,
     double p[kMaxLevels], delta[kMaxLevels];
     if (adaptive || need_delta) {
         for (int l = 0; l < sc.L; ++l) {
-            // exact 128-bit sum of the per-block partials, rounded once to fp64
+            // exact 128-bit sum of the per-block partials (lanes take every 32nd, integer adds: any order),
+            // rounded once to fp64
             unsigned __int128 S = 0;
-            for (int c = 0; c < n_partials; ++c) S += S_partial[((int64_t)m * stat_ctas + c) * kMaxLevels + l];
-            const double Sd = (double)(unsigned long long)(S >> 64) * 0x1.0p64 + (double)(unsigned long long)S;
+            for (int c = lane; c < n_partials; c += 32) S += S_partial[((int64_t)m * stat_ctas + c) * kMaxLevels + l];
+            unsigned long long lo = (unsigned long long)S, hi = (unsigned long long)(S >> 64);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long lo2 = __shfl_xor_sync(0xFFFFFFFFu, lo, o), hi2 = __shfl_xor_sync(0xFFFFFFFFu, hi, o);
+                const unsigned __int128 t = (((unsigned __int128)hi << 64) | lo) + (((unsigned __int128)hi2 << 64) | lo2);
+                lo = (unsigned long long)t;
+                hi = (unsigned long long)(t >> 64);
+            }
+            const double Sd = (double)hi * 0x1.0p64 + (double)lo;
             delta[l] = (double)gmax * ldexp(1.0, -sc.bits[l]) * sqrt(Sd);
-            delta_all[m * kMaxLevels + l] = delta[l];
         }
     }
+    if (lane != 0) return;
+    if (adaptive || need_delta)
+        for (int l = 0; l < sc.L; ++l) delta_all[m * kMaxLevels + l] = delta[l];
     if (adaptive) {
         double s = 0.0;
         for (int l = 0; l < sc.L; ++l) s += delta[l];
@@ -307,38 +321,62 @@ aggregate_bitwise_kernel(const uint32_t* __restrict__ planes, const float* __res
                          int w_max, int64_t words, int M, int64_t d, float* __restrict__ out) {
     __shared__ float sh_out[kBitThreads / 32][32][33];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float fM = (float)M;
+    const float inv_M = 1.0f / (float)M;
     const int64_t nblk = (words + kBitThreads - 1) / kBitThreads;
     for (int64_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
         const int64_t word = blk * kBitThreads + threadIdx.x;
         float acc[32];
 #pragma unroll
         for (int t = 0; t < 32; ++t) acc[t] = 0.0f;
+        // the sign word and the first magnitude plane of the next worker are loaded before this worker's are used
+        uint32_t sgn_n = 0, pw1_n = 0;
+        auto preload = [&](int mm) {
+            if (mm < M && level[mm] >= 0 && word < words) {
+                const uint32_t* pm = planes + (int64_t)mm * (1 + w_max) * words;
+                sgn_n = pm[word];
+                pw1_n = pm[words + word];
+            } else {
+                sgn_n = 0;
+                pw1_n = 0;
+            }
+        };
+        preload(0);
         for (int m = 0; m < M; ++m) {  // fixed worker order
             const int lv = level[m];
+            const uint32_t sgn = sgn_n, pw1 = pw1_n;
+            preload(m + 1);
             if (lv < 0) continue;
             const int w = sc.width[lv];
             // value of one unit of the field: 2^{-b_l} gmax / p_l
             const float unit = (float)(ldexp((double)gmax[m], -sc.bits[lv]) / p_sel[m]);
-            const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
-            const uint32_t sgn = (word < words) ? pm[word] : 0u;
-            uint32_t f[32];
+            if (w == 1) {  // the paper's case: one information bit and one sign bit per entry
+                const uint32_t ub = __float_as_uint(unit);
 #pragma unroll
-            for (int t = 0; t < 32; ++t) f[t] = 0;
-            for (int j = 1; j <= w; ++j) {
-                const uint32_t pw = (word < words) ? pm[(int64_t)j * words + word] : 0u;
+                for (int t = 0; t < 32; ++t) {
+                    const uint32_t on = 0u - ((pw1 >> t) & 1u);
+                    acc[t] += __uint_as_float((ub & on) ^ (((sgn >> t) & 1u) << 31));
+                }
+            } else {
+                const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
+                uint32_t f[32];
 #pragma unroll
-                for (int t = 0; t < 32; ++t) f[t] = (f[t] << 1) | ((pw >> t) & 1u);
-            }
+                for (int t = 0; t < 32; ++t) f[t] = (pw1 >> t) & 1u;
+                for (int j = 2; j <= w; ++j) {
+                    const uint32_t pw = (word < words) ? pm[(int64_t)j * words + word] : 0u;
 #pragma unroll
-            for (int t = 0; t < 32; ++t) {
-                const float v = (float)f[t] * unit;
-                acc[t] += ((sgn >> t) & 1u) ? -v : v;
+                    for (int t = 0; t < 32; ++t) f[t] = (f[t] << 1) | ((pw >> t) & 1u);
+                }
+#pragma unroll
+                for (int t = 0; t < 32; ++t) {
+                    // f < 2^23: exact integer-to-float through the 2^23 offset, without the conversion unit
+                    const float ff = __uint_as_float(0x4B000000u | f[t]) - 8388608.0f;
+                    acc[t] += __uint_as_float(__float_as_uint(ff * unit) ^ (((sgn >> t) & 1u) << 31));
+                }
             }
         }
         // transpose through shared memory so that the 32 floats of a word leave as one 128-byte row
 #pragma unroll
-        for (int t = 0; t < 32; ++t) sh_out[warp][lane][t] = acc[t] / fM;
+        for (int t = 0; t < 32; ++t) sh_out[warp][lane][t] = acc[t] * inv_M;
         __syncwarp();
         const int64_t wbase = blk * kBitThreads + warp * 32;
 #pragma unroll 4
@@ -416,6 +454,7 @@ void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M,
     cudaMemsetAsync(ws.S_partial, 0, (size_t)M * ws.stat_ctas * kMaxLevels * sizeof(unsigned long long), s);
     int nb = bit_blocks(ws, d, dtype == MLMC_BF16 ? 8 : 4, M, 4);
     if (nb > ws.stat_ctas) nb = ws.stat_ctas;
+    ws.cur_stat_ctas = nb;
     LaunchScope t(ws, K_BIT_STATS, s);
     if (dtype == MLMC_BF16)
         launch_bit_stats_t<bf16_t>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, nb, s);
@@ -427,8 +466,8 @@ void launch_bit_probs_draw(Workspace& ws, int M, const int32_t* b, int L, bool a
                            uint64_t seed, uint64_t step, const mlmc_bit_msgs* out, cudaStream_t s) {
     const BitSchedule sc = make_schedule(b, L);
     LaunchScope t(ws, K_BIT_DRAW, s);
-    bit_probs_draw_kernel<<<(M + 63) / 64, 64, 0, s>>>(
-        sc, ws.gmax_bits, ws.S_partial, ws.stat_ctas, ws.stat_ctas, ws.p_fixed, adaptive ? 1 : 0, need_delta ? 1 : 0,
+    bit_probs_draw_kernel<<<M, 32, 0, s>>>(
+        sc, ws.gmax_bits, ws.S_partial, ws.cur_stat_ctas, ws.stat_ctas, ws.p_fixed, adaptive ? 1 : 0, need_delta ? 1 : 0,
         seed, step, M, ws.p_all, ws.delta_all, ws.u_dev, ws.bit_level, out ? out->gmax : nullptr,
         out ? out->level : nullptr, out ? out->p_sel : nullptr, out ? out->w_max : 0, out ? 1 : 0, ws.status,
         ws.worker_err);

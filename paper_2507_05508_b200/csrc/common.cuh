@@ -102,7 +102,7 @@ struct Workspace {
     // bit-wise
     uint32_t* gmax_bits;         // [M]
     unsigned long long* S_partial;  // [M][stat_ctas][kMaxLevels]
-    int stat_ctas;
+    int stat_ctas, cur_stat_ctas;
     int32_t* bit_level;          // [M] (mirrors out->level for the pack kernel)
 };
 
