@@ -1,0 +1,134 @@
+"""Parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times.
+
+The oracle cannot sort eight 124M-entry rows in reasonable time, so per workload
+  * one worker's whole row goes through the oracle and is compared element by element
+    (level, probability, every band index, every value; bit planes for the bit-wise path),
+  * every worker is checked through properties that hold at any size: the message has exactly
+    k_l - k_{l-1} entries, indices strictly ascending, values = g_i / p_l within 1e-6, and the band is a
+    rank interval: fewer than k_l entries of the row are larger than its smallest member, at most k_{l-1}
+    are larger than its largest one,
+  * the dense mean is compared with the oracle's average of the emitted messages on every coordinate.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_05508_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+VAL_RTOL = 1e-6
+AGG_RTOL = 1e-6
+MARGIN = 1e-9
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2507_05508_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _topk_fullsize(B, ora, w, step, oracle_workers=(0,)):
+    torch.cuda.set_device(0)
+    k = wl.topk_schedule(w)
+    L = len(k)
+    p = None if w.adaptive else list(wl.geometric_probs(L))
+    ctx = B.mlmc_create(0, w.d, w.M, 32)           # as bench.py's Runner does
+    try:
+        g = wl.gradients(w, step, "cuda")
+        out = B.TopkBuffers(w.M, wl.max_band(k))
+        dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+        B.mlmc_compress_topk(ctx, g, k, p, w.seed, step, out)
+        B.mlmc_aggregate(ctx, B.MLMC_TOPK, out, None, w.M, w.d, dense)
+        assert B.mlmc_get_status(ctx) == B.MLMC_OK
+        level, count, p_sel = out.level.tolist(), out.count.tolist(), out.p_sel.tolist()
+        kk = [0] + list(k)
+        msgs = []
+        for m in range(w.M):
+            l, n = level[m], count[m]
+            assert 0 <= l < L and n == kk[l + 1] - kk[l]
+            idx = out.idx[m, :n].to(torch.int64) & 0xFFFFFFFF
+            val = out.val[m, :n]
+            if n > 1:
+                assert bool((idx[1:] > idx[:-1]).all())                  # strictly ascending, hence unique
+            if n:
+                assert int(idx[-1]) < w.d
+                mag = g[m].float().abs()
+                band = mag[idx]
+                ref = (g[m].float()[idx].double() / p_sel[m])
+                assert bool(((val.double() - ref).abs() <= VAL_RTOL * ref.abs()).all())
+                lo, hi = band.min(), band.max()
+                assert int((mag > lo).sum()) < kk[l + 1] <= int((mag >= lo).sum())
+                assert int((mag > hi).sum()) <= kk[l] < int((mag >= hi).sum())
+                del mag, band, ref
+            msgs.append((out.idx[m, :n].cpu().numpy().view(np.uint32), out.val[m, :n].cpu().numpy()))
+        for m in oracle_workers:                                         # whole rows through the oracle
+            row = wl.as_numpy_bits(g[m:m + 1])[0]
+            o = ora.topk(row, k, p=p, seed=w.seed, step=step, worker=m)
+            if o.margin < MARGIN and level[m] != o.level:
+                o = ora.topk(row, k, p=p, seed=w.seed, step=step, worker=m, force_level=level[m])
+            assert level[m] == o.level
+            assert abs(p_sel[m] - o.p_sel) <= 1e-10 * o.p_sel
+            assert np.array_equal(msgs[m][0], o.idx)
+            assert np.all(np.abs(msgs[m][1].astype(np.float64) - o.val) <= VAL_RTOL * np.abs(o.val))
+        ref, scale = ora.aggregate_topk(msgs, w.d)
+        got = dense.cpu().numpy().astype(np.float64)
+        assert not np.isnan(got).any()
+        assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
+    finally:
+        B.mlmc_destroy(ctx)
+
+
+def test_c3_full_size(B, ora):
+    _topk_fullsize(B, ora, wl.C3, step=0, oracle_workers=(0, 15))
+
+
+def test_c4_full_size(B, ora):
+    _topk_fullsize(B, ora, wl.C4, step=1, oracle_workers=(31,))
+
+
+def test_c5a_full_size(B, ora):
+    _topk_fullsize(B, ora, wl.C5A, step=0, oracle_workers=(3,))
+
+
+def test_c5b_full_size(B, ora):
+    w = wl.C5B
+    torch.cuda.set_device(0)
+    b = list(w.bits)
+    widths = np.diff(np.concatenate([[0], b]))
+    ctx = B.mlmc_create(0, w.d, w.M, 32)
+    try:
+        g = wl.gradients(w, 0, "cuda")
+        out = B.BitBuffers(w.M, w.d, int(widths.max()))
+        dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+        B.mlmc_compress_bitwise(ctx, g, b, None, w.seed, 0, out)
+        B.mlmc_aggregate(ctx, B.MLMC_BITWISE, out, b, w.M, w.d, dense)
+        assert B.mlmc_get_status(ctx) == B.MLMC_OK
+        level, p_sel, gmax = out.level.tolist(), out.p_sel.tolist(), out.gmax.cpu().numpy()
+        assert np.array_equal(gmax, g.abs().max(dim=1).values.cpu().numpy())       # the normaliser of every worker
+
+        class Msg:
+            pass
+
+        msgs = []
+        for m in range(w.M):
+            mm = Msg()
+            wv = int(widths[level[m]])
+            mm.planes = out.planes[m, :1 + wv].cpu().numpy().view(np.uint32)
+            mm.gmax, mm.level, mm.p_sel = float(gmax[m]), level[m], p_sel[m]
+            msgs.append(mm)
+        for m in (0, 5):                                                   # whole rows through the oracle
+            row = wl.as_numpy_bits(g[m:m + 1])[0]
+            o = ora.bitwise(row, b, None, seed=w.seed, step=0, worker=m)
+            if o.margin < MARGIN and level[m] != o.level:
+                o = ora.bitwise(row, b, None, seed=w.seed, step=0, worker=m, force_level=level[m])
+            assert level[m] == o.level and np.float32(o.gmax) == gmax[m]
+            assert abs(p_sel[m] - o.p_sel) <= 1e-10 * o.p_sel
+            assert np.array_equal(msgs[m].planes, o.planes)
+        ref, scale = ora.aggregate_bitwise(msgs, b, w.d)
+        got = dense.cpu().numpy().astype(np.float64)
+        assert not np.isnan(got).any()
+        assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
+    finally:
+        B.mlmc_destroy(ctx)
