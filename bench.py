@@ -1,11 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the MLMC compress+aggregate hot path.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5a] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl reference]
 
 One step = mlmc_compress_* on all M workers + mlmc_aggregate into the dense mean, on one batch of
-synthetic gradients already resident in HBM.  `value` is gradient GB/s = M*d*sizeof(T) / step time,
-summed over ranks (ranks are independent replicas: the path has no inter-GPU exchange).
+synthetic gradients already resident in HBM.  The default workload c5 is the 124M-parameter config with
+both of its variants per step (adaptive MLMC-Top-k, then adaptive bit-wise MLMC, each a full
+compress + aggregate over the same gradient batch).  `value` is gradient GB/s = gradient bytes swept by
+the variants (M*d*sizeof(T) each) / step time, summed over ranks (ranks are independent replicas: the
+path has no inter-GPU exchange).
 Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
@@ -37,7 +40,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c5a", choices=["c1", "c2", "c3", "c4", "c5a", "c5b"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c5a", "c5b"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -57,6 +60,18 @@ def measured_peak():
 
 def elem_size(w):
     return 2 if w.dtype == "bf16" else 4
+
+
+def sub_workloads(name: str):
+    """The variants one step runs: c5 is both the Top-k and the bit-wise variant of the 124M config."""
+    from paper_2507_05508_b200 import workloads as wl
+    return [wl.C5A, wl.C5B] if name == "c5" else [wl.ALL[name]]
+
+
+def describe(subs) -> str:
+    w = subs[0]
+    kinds = " + ".join(f"{'adaptive' if x.adaptive else 'fixed-p'} MLMC-{x.kind}" for x in subs)
+    return f"{'c5' if len(subs) == 2 else w.name}: {kinds}, d={w.d}, M={w.M}, {w.dtype}"
 
 
 # --------------------------------------------------------------------------------------------------
@@ -145,13 +160,14 @@ class ClockSampler:
 # the CUDA arm
 # --------------------------------------------------------------------------------------------------
 class Runner:
-    """Owns the buffers of one workload and runs steps through the C ABI."""
+    """Owns the buffers of one workload (one or two variants over the same batch) and runs steps through the C ABI."""
 
-    def __init__(self, w, device_index: int, n_batches: int = 2, rank: int = 0):
+    def __init__(self, subs, device_index: int, n_batches: int = 2, rank: int = 0):
         import torch
         from paper_2507_05508_b200 import binding as B
         from paper_2507_05508_b200 import workloads as wl
-        self.torch, self.B, self.wl, self.w = torch, B, wl, w
+        self.torch, self.B, self.wl, self.subs = torch, B, wl, subs
+        w = self.w = subs[0]
         self.dev = f"cuda:{device_index}"
         torch.cuda.set_device(device_index)
         self.ctx = B.mlmc_create(device_index, w.d, w.M, 32)
@@ -159,35 +175,41 @@ class Runner:
         self.batches = [wl.gradients(w, 1000 * rank + i, self.dev, sc) for i in range(n_batches)]
         del sc
         self.dense = torch.empty(w.d, dtype=torch.float32, device=self.dev)
-        if w.kind == "topk":
-            self.k = wl.topk_schedule(w)
-            self.L = len(self.k)
-            self.msgs = B.TopkBuffers(w.M, wl.max_band(self.k), self.dev)
-        else:
-            self.b = list(w.bits)
-            self.L = len(self.b)
-            widths = [self.b[0]] + [self.b[i] - self.b[i - 1] for i in range(1, self.L)]
-            self.msgs = B.BitBuffers(w.M, w.d, max(widths), self.dev)
-        self.p = None if w.adaptive else list(wl.geometric_probs(self.L))
+        self.plan = []
+        for x in subs:
+            if x.kind == "topk":
+                sched = wl.topk_schedule(x)
+                msgs = B.TopkBuffers(x.M, wl.max_band(sched), self.dev)
+            else:
+                sched = list(x.bits)
+                widths = [sched[0]] + [sched[i] - sched[i - 1] for i in range(1, len(sched))]
+                msgs = B.BitBuffers(x.M, x.d, max(widths), self.dev)
+            p = None if x.adaptive else list(wl.geometric_probs(len(sched)))
+            self.plan.append((x, sched, p, msgs))
+        self.L = [len(pl[1]) for pl in self.plan]
         torch.cuda.synchronize()
 
     def step(self, i: int, g=None):
-        B, w = self.B, self.w
+        B = self.B
         g = self.batches[i % len(self.batches)] if g is None else g
-        if w.kind == "topk":
-            B.mlmc_compress_topk(self.ctx, g, self.k, self.p, w.seed, i, self.msgs)
-            B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, self.msgs, None, w.M, w.d, self.dense)
-        else:
-            B.mlmc_compress_bitwise(self.ctx, g, self.b, self.p, w.seed, i, self.msgs)
-            B.mlmc_aggregate(self.ctx, B.MLMC_BITWISE, self.msgs, self.b, w.M, w.d, self.dense)
+        for x, sched, p, msgs in self.plan:
+            if x.kind == "topk":
+                B.mlmc_compress_topk(self.ctx, g, sched, p, x.seed, i, msgs)
+                B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, self.dense)
+            else:
+                B.mlmc_compress_bitwise(self.ctx, g, sched, p, x.seed, i, msgs)
+                B.mlmc_aggregate(self.ctx, B.MLMC_BITWISE, msgs, sched, x.M, x.d, self.dense)
 
-    def message_bytes(self) -> float:
-        """Bytes of the messages of the last step (written once by compress, read once by aggregate)."""
-        if self.w.kind == "topk":
-            return float(self.msgs.count.sum().item()) * 8.0
-        widths = [self.b[0]] + [self.b[i] - self.b[i - 1] for i in range(1, self.L)]
-        lv = self.msgs.level.tolist()
-        return float(sum((1 + widths[l]) * self.msgs.words * 4 for l in lv if l >= 0))
+    def message_bytes(self):
+        """Per variant kind: bytes of the messages of the last step (written once by compress, read once by aggregate)."""
+        out = {}
+        for x, sched, p, msgs in self.plan:
+            if x.kind == "topk":
+                out["topk"] = float(msgs.count.sum().item()) * 8.0
+            else:
+                widths = [sched[0]] + [sched[i] - sched[i - 1] for i in range(1, len(sched))]
+                out["bitwise"] = float(sum((1 + widths[l]) * msgs.words * 4 for l in msgs.level.tolist() if l >= 0))
+        return out
 
     def close(self):
         self.B.mlmc_destroy(self.ctx)
@@ -201,12 +223,13 @@ def sweeps_charged(w) -> int:
     return 3 if w.adaptive else 2
 
 
-# Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes, dense bytes).
-def kernel_alg_bytes(name: str, sweep: float, msg: float, dense: float):
+# Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes of its variant, dense bytes).
+def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float):
+    mt, mb = msg.get("topk", 0.0), msg.get("bitwise", 0.0)
     table = {
         "hist1": sweep, "sums_candidates": sweep, "masked_pass2": sweep, "masked_pass3": sweep, "norm_sweep": sweep,
-        "emit": sweep + msg, "aggregate_topk": msg + dense,
-        "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + msg, "aggregate_bitwise": msg + dense,
+        "emit": sweep + mt, "aggregate_topk": mt + dense,
+        "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + mb, "aggregate_bitwise": mb + dense,
     }
     return table.get(name)
 
@@ -217,11 +240,12 @@ def run_cuda(args):
     from paper_2507_05508_b200 import workloads as wl
     cuda_build.build()
     rank, world, local = dist_setup(args.gpus)
-    w = wl.ALL[args.workload]
+    subs = sub_workloads(args.workload)
     if args.shrink_d or args.shrink_M:
-        w = wl.shrink(w, args.shrink_d or w.d, args.shrink_M or w.M)
+        subs = [wl.shrink(x, args.shrink_d or x.d, args.shrink_M or x.M) for x in subs]
+    w = subs[0]
     peak, peak_kind = measured_peak()
-    r = Runner(w, local, rank=rank)
+    r = Runner(subs, local, rank=rank)
     B = r.B
     sweep_bytes = float(w.M) * w.d * elem_size(w)
     dense_bytes = float(w.d) * 4.0
@@ -234,7 +258,7 @@ def run_cuda(args):
     # ---- timed region: exactly K steps, device-timed, per-kernel event pairs on the same stream
     B.mlmc_timing_enable(r.ctx, True)
     launches0 = B.mlmc_launch_count(r.ctx)
-    msg_bytes_total = 0.0
+    msg_acc = {}
     sampler = ClockSampler(local)
     barrier(world)
     torch.cuda.synchronize()
@@ -255,19 +279,21 @@ def run_cuda(args):
     B.mlmc_timing_enable(r.ctx, False)
     status = B.mlmc_get_status(r.ctx)
     ms_per_step = total_ms / args.steps
-    value = world * sweep_bytes / (ms_per_step * 1e-3) / 1e9
+    value = world * len(subs) * sweep_bytes / (ms_per_step * 1e-3) / 1e9
 
     # message volume: average over a few steps outside the timed region (levels are redrawn every step)
     probe = min(args.steps, 8)
     for i in range(probe):
         r.step(args.warmup + i)
-        msg_bytes_total += r.message_bytes()
-    msg_bytes = msg_bytes_total / probe
+        for kind, v in r.message_bytes().items():
+            msg_acc[kind] = msg_acc.get(kind, 0.0) + v
+    msg_by_kind = {kind: v / probe for kind, v in msg_acc.items()}
+    msg_bytes = sum(msg_by_kind.values())
 
     # ---- roofline of the dominant kernel and of the whole step
     dom = max(per_kernel.items(), key=lambda kv: kv[1][0])
     dom_name, (dom_ms, dom_n) = dom
-    dom_bytes = kernel_alg_bytes(dom_name, sweep_bytes, msg_bytes, dense_bytes) or sweep_bytes
+    dom_bytes = kernel_alg_bytes(dom_name, sweep_bytes, msg_by_kind, dense_bytes) or sweep_bytes
     dom_avg_s = dom_ms / dom_n * 1e-3
     achieved = dom_bytes / dom_avg_s / 1e9
     ratio = NCU_TRAFFIC_RATIO.get(f"{dom_name}:{w.dtype}")
@@ -275,7 +301,7 @@ def run_cuda(args):
                 "frac": round(achieved / peak, 4), "peak_source": peak_kind,
                 "traffic": None if ratio is None else ratio * dom_bytes,
                 "alg_bytes_per_launch": dom_bytes, "avg_launch_ms": round(dom_avg_s * 1e3, 4)}
-    b_alg = sweeps_charged(w) * sweep_bytes + 2 * msg_bytes + dense_bytes
+    b_alg = sum(sweeps_charged(x) * sweep_bytes + dense_bytes for x in subs) + 2 * msg_bytes
     step_frac = b_alg / (ms_per_step * 1e-3) / 1e9 / peak
     kernels = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] / args.steps,
                    "share": round(v[0] / sum(x[0] for x in per_kernel.values()), 4)}
@@ -305,14 +331,14 @@ def run_cuda(args):
         torch.cuda.synchronize()
         barrier(world)
         e2e_ms = max_over_ranks(a.elapsed_time(b), world, r.dev) / args.e2e_steps
-        e2e = {"value": round(world * sweep_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
+        e2e = {"value": round(world * len(subs) * sweep_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
                "h2d_bytes_per_step": int(sweep_bytes), "d2h_bytes_per_step": int(dense_bytes),
                "ms_per_step": round(e2e_ms, 3)}
         del host_in, host_out
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(w, r.batches[0][0], budget_s=15.0)
+        cpu = cpu_baseline(subs, r.batches[0][0], budget_s=15.0)
 
     if rank == 0:
         line = {
@@ -320,11 +346,10 @@ def run_cuda(args):
             "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16",
             "data": "synthetic",
-            "config": {"workload": f"{w.name}: {'adaptive' if w.adaptive else 'fixed-p'} MLMC-{w.kind}, d={w.d}, "
-                                   f"M={w.M}, {w.dtype}, L={r.L}", "l2_policy": "inputs larger than L2: "
+            "config": {"workload": describe(subs) + f", L={r.L}", "l2_policy": "inputs larger than L2: "
                        f"{sweep_bytes / 1e6:.0f} MB per sweep, 2 batches alternated", "parallelism": "replicas only"},
-            "elements_per_s": round(world * w.M * w.d / (ms_per_step * 1e-3), 1),
-            "step_roofline": {"alg_bytes_per_step": b_alg, "sweeps_charged": sweeps_charged(w),
+            "elements_per_s": round(world * len(subs) * w.M * w.d / (ms_per_step * 1e-3), 1),
+            "step_roofline": {"alg_bytes_per_step": b_alg, "sweeps_charged": [sweeps_charged(x) for x in subs],
                               "message_bytes_per_step": msg_bytes, "frac_of_peak": round(step_frac, 4),
                               "frac_of_8TBs": round(b_alg / (ms_per_step * 1e-3) / 8e12, 4)},
             "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "e2e": e2e,
@@ -340,48 +365,51 @@ def run_cuda(args):
 # --------------------------------------------------------------------------------------------------
 # the oracle, timed on the host cores (reported baseline, and the --impl reference arm)
 # --------------------------------------------------------------------------------------------------
-def oracle_sample_step(w, g_row_np, d_s: int, step: int):
-    """One worker's compress + its aggregate share on the first d_s coordinates; returns seconds."""
+def oracle_sample_step(subs, g_row_np, d_s: int, step: int):
+    """One worker's compress + its aggregate share on the first d_s coordinates, for every variant; returns seconds."""
     import numpy as np
     import oracle
     from paper_2507_05508_b200 import workloads as wl
     x = np.ascontiguousarray(g_row_np[:d_s])
     t0 = time.perf_counter()
-    if w.kind == "topk":
-        ws = wl.shrink(w, d_s, 1)
-        k = wl.topk_schedule(ws)
-        p = None if w.adaptive else wl.geometric_probs(len(k))
-        m = oracle.topk(x, k, p=p, seed=w.seed, step=step, worker=0)
-        oracle.aggregate_topk([(m.idx, m.val)], d_s)
-    else:
-        b = list(w.bits)
-        p = None if w.adaptive else wl.geometric_probs(len(b))
-        m = oracle.bitwise(x, b, p=p, seed=w.seed, step=step, worker=0)
-        oracle.aggregate_bitwise([m], b, d_s)
+    for w in subs:
+        if w.kind == "topk":
+            ws = wl.shrink(w, d_s, 1)
+            k = wl.topk_schedule(ws)
+            p = None if w.adaptive else wl.geometric_probs(len(k))
+            m = oracle.topk(x, k, p=p, seed=w.seed, step=step, worker=0)
+            oracle.aggregate_topk([(m.idx, m.val)], d_s)
+        else:
+            b = list(w.bits)
+            p = None if w.adaptive else wl.geometric_probs(len(b))
+            m = oracle.bitwise(x, b, p=p, seed=w.seed, step=step, worker=0)
+            oracle.aggregate_bitwise([m], b, d_s)
     return time.perf_counter() - t0
 
 
-def calibrate_sample(w, g_row_np, budget_s: float) -> int:
+def calibrate_sample(subs, g_row_np, budget_s: float) -> int:
     """Largest power-of-two prefix whose oracle step fits the per-step budget (extrapolated from a probe)."""
-    probe = min(1 << 18, w.d)
-    t = max(oracle_sample_step(w, g_row_np, probe, 0), 1e-4)
+    d = subs[0].d
+    probe = min(1 << 18, d)
+    t = max(oracle_sample_step(subs, g_row_np, probe, 0), 1e-4)
     d_s = probe
-    while d_s * 2 <= min(w.d, 1 << 25) and t * 2.2 <= budget_s:
+    while d_s * 2 <= min(d, 1 << 25) and t * 2.2 <= budget_s:
         d_s *= 2
         t *= 2.2
     return d_s
 
 
-def cpu_baseline(w, g_row, budget_s: float):
+def cpu_baseline(subs, g_row, budget_s: float):
     import oracle
     from paper_2507_05508_b200 import workloads as wl
     oracle.build()
+    w = subs[0]
     row = wl.as_numpy_bits(g_row.unsqueeze(0))[0]
-    d_s = calibrate_sample(w, row, budget_s)
-    t = oracle_sample_step(w, row, d_s, 1)
-    return {"value": round(d_s * elem_size(w) / t / 1e9, 5), "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"1 worker, first {d_s} of d={w.d} coordinates, compress + aggregate, {t:.2f} s",
-            "elements_per_s": round(d_s / t, 1)}
+    d_s = calibrate_sample(subs, row, budget_s)
+    t = oracle_sample_step(subs, row, d_s, 1)
+    return {"value": round(len(subs) * d_s * elem_size(w) / t / 1e9, 5), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"1 worker, first {d_s} of d={w.d} coordinates, compress + aggregate of every variant, {t:.2f} s",
+            "elements_per_s": round(len(subs) * d_s / t, 1)}
 
 
 def run_reference(args):
@@ -393,27 +421,28 @@ def run_reference(args):
     import oracle
     from paper_2507_05508_b200 import workloads as wl
     oracle.build()
-    w = wl.ALL[args.workload]
+    subs = sub_workloads(args.workload)
+    w = subs[0]
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     d_gen = min(w.d, 1 << 25)
     wg = wl.shrink(w, d_gen, 1) if d_gen < w.d else w
     row = wl.as_numpy_bits(wl.gradients(wg, 0, dev)[:1])[0]
     per_step_budget = max(0.05, 150.0 / max(1, args.steps + args.warmup))
-    d_s = min(calibrate_sample(w, row, per_step_budget), d_gen)
+    d_s = min(calibrate_sample(subs, row, per_step_budget), d_gen)
     for i in range(args.warmup):
-        oracle_sample_step(w, row, d_s, i)
+        oracle_sample_step(subs, row, d_s, i)
     t0 = time.perf_counter()
     for i in range(args.steps):
-        oracle_sample_step(w, row, d_s, args.warmup + i)
+        oracle_sample_step(subs, row, d_s, args.warmup + i)
     t = (time.perf_counter() - t0) / args.steps
-    value = d_s * elem_size(w) / t / 1e9
-    sample = f"each step: 1 worker, first {d_s} of d={w.d} coordinates, compress + aggregate on 1 host core"
+    value = len(subs) * d_s * elem_size(w) / t / 1e9
+    sample = (f"each step: 1 worker, first {d_s} of d={w.d} coordinates, compress + aggregate of every variant "
+              "on 1 host core")
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": UNIT,
             "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(t * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if w.dtype == "f32" else "bf16", "data": "synthetic",
-            "config": {"workload": f"{w.name}: {'adaptive' if w.adaptive else 'fixed-p'} MLMC-{w.kind}, d={w.d}, "
-                                   f"M={w.M}, {w.dtype}", "sample": sample},
+            "config": {"workload": describe(subs), "sample": sample},
             "cpu_baseline": {"value": round(value, 5), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 5), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
