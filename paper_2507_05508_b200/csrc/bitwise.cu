@@ -24,12 +24,35 @@ struct BitSchedule {
     int bits[kMaxLevels];       // b_l
 };
 
-__device__ __forceinline__ uint32_t fixed_point_code(float mag, float gmax, float two_b, uint32_t qmax) {
-    const float e = __fdiv_rn(mag, gmax);        // IEEE division: "divide the entries by the largest entry"
-    const float scaled = __fmul_rn(e, two_b);    // exact power-of-two scaling
-    const uint32_t q = __float2uint_rz(scaled);  // truncation: the lower bits are discarded
-    return min(q, qmax);
-}
+// The code q = min(trunc(fl32(|g| / gmax) * 2^B), 2^B - 1) with the IEEE-rounded fp32 quotient, for a fixed
+// divisor.  The quotient is formed in fp64 as |g| * (1 / gmax) and rounded to fp32 once: a quotient of two
+// 24-bit significands is never closer than 2^-49 (relative) to the midpoint of two fp32 numbers, the fp64
+// product is within 2^-52 of it, so this rounding is the same as that of the fp32 division.
+struct Quantiser {
+    double inv;     // fl64(1 / gmax)
+    float gmax;
+    float two_b;    // 2^B
+    uint32_t qmax;  // 2^B - 1
+    bool widen_by_bits;  // gmax >= 2^-100: an fp32 operand below the normal range cannot reach q = 1, so its
+                         // fp64 image may be built from the bit pattern as if it were normal
+    __device__ __forceinline__ Quantiser(float g, int B) {
+        inv = g > 0.0f ? 1.0 / (double)g : 0.0;
+        gmax = g;
+        two_b = (float)(1u << B);
+        qmax = (1u << B) - 1u;
+        widen_by_bits = g >= 0x1.0p-100f;
+    }
+    __device__ __forceinline__ uint32_t code(uint32_t mag_bits /* sign bit cleared */) const {
+        double x;
+        if (widen_by_bits)
+            x = __hiloint2double((int)((mag_bits >> 3) + 0x38000000u), (int)(mag_bits << 29));
+        else
+            x = (double)__uint_as_float(mag_bits);
+        const float e = (float)(x * inv);              // = fl32(|g| / gmax)
+        const float scaled = __fmul_rn(e, two_b);      // exact power-of-two scaling
+        return min(__float2uint_rz(scaled), qmax);     // truncation: the lower bits are discarded
+    }
+};
 
 // ---- per-worker max |g| as an integer max over magnitude keys; flags NaN / Inf
 template <typename T>
@@ -90,8 +113,7 @@ bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t*
     const int m = blockIdx.y;
     if (worker_err[m]) return;
     const float gmax = __uint_as_float(gmax_bits[m]);
-    const float two_b = (float)(1u << sc.B);
-    const uint32_t qmax = (1u << sc.B) - 1u;
+    const Quantiser qz(gmax, sc.B);
     unsigned long long acc[LMAX];
     int sh[LMAX];
     uint32_t mk[LMAX];
@@ -106,8 +128,7 @@ bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t*
         int64_t v0, v1;
         block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
         auto take = [&](uint32_t bits) {
-            const float mag = fabsf(Tr::value(bits));
-            const uint32_t q = fixed_point_code(mag, gmax, two_b, qmax);
+            const uint32_t q = qz.code(__float_as_uint(Tr::value(bits)) & 0x7FFFFFFFu);
 #pragma unroll
             for (int l = 0; l < LMAX; ++l) {
                 const uint32_t f = (q >> sh[l]) & mk[l];
@@ -251,8 +272,7 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
     const int warps_per_block = kBitThreads / 32;
     const int64_t ngroups = (words + 31) / 32;  // groups of 32 words = 1024 entries
     const float gmax = __uint_as_float(gmax_bits[m]);
-    const float two_b = (float)(1u << sc.B);
-    const uint32_t qmax = (1u << sc.B) - 1u;
+    const Quantiser qz(gmax, sc.B);
     const int shift = sc.shift[level];
     const uint32_t mask = sc.mask[level];
     const int w = sc.width[level];
@@ -295,7 +315,7 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
             else
                 bits = reinterpret_cast<const uint16_t*>(buf)[s * 32 + lane];
             const float x = Tr::value(bits);
-            const uint32_t q = (gmax > 0.0f) ? fixed_point_code(fabsf(x), gmax, two_b, qmax) : 0u;
+            const uint32_t q = (gmax > 0.0f) ? qz.code(__float_as_uint(x) & 0x7FFFFFFFu) : 0u;
             code[s] = ((q >> shift) & mask) | (__float_as_uint(x) & 0x80000000u);
         }
         const int64_t word = grp * 32 + lane;
