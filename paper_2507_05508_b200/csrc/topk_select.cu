@@ -249,10 +249,11 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is
 // sweep 2 (fp32): per-interval energy of the bins that hold no threshold, and compaction of the keys
 // of the bins that do ("candidates": a few percent of the data) for the remaining digit passes
 // -------------------------------------------------------------------------------------------
-constexpr int kS2Threads = 256;
-constexpr int kS2Vecs = 4;                                   // 16-byte vectors per thread per round
+constexpr int kS2Threads = 512;
+constexpr int kS2Vecs = 2;                                   // 16-byte vectors per thread per round
 constexpr int kS2Round = kS2Threads * kS2Vecs * 4;            // elements per round
-constexpr int kStage = 2 * kS2Round;                          // staged candidate keys per block
+constexpr int kStageSlack = 1024;                             // candidates that may wait for the next flush
+constexpr int kStage = kS2Round + kStageSlack;                // staged candidate keys per block
 
 // table: bin -> code.  code < 64: the bin lies wholly inside open interval `code` (between two thresholds);
 // code >= 64: the bin may hold a threshold, its keys are compacted into the candidate buffer.
@@ -347,7 +348,7 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
             }
         }
         __syncthreads();
-        if (sh_n > (uint32_t)(kStage - kS2Round)) flush();  // uniform: sh_n is read after the barrier
+        if (sh_n > (uint32_t)kStageSlack) flush();  // uniform: sh_n is read after the barrier; a round adds at most kS2Round
 #pragma unroll
         for (int j = 0; j < kS2Vecs; ++j) cur[j] = nxt[j];
     }
