@@ -81,7 +81,7 @@ typedef struct {
 } mlmc_bit_msgs;
 
 /* Allocates the scratch workspace for problems up to (d_max, M_max, L_max) on `device`.
- * Synchronous.  L_max <= MLMC_MAX_LEVELS.  Returns MLMC_ERR_NOMEM / MLMC_ERR_CUDA on failure. */
+ * Synchronous.  L_max <= MLMC_MAX_LEVELS, M_max <= 1024.  Returns MLMC_ERR_NOMEM / MLMC_ERR_CUDA on failure. */
 int mlmc_create(mlmc_ctx** ctx, int device, int64_t d_max, int M_max, int L_max);
 int mlmc_destroy(mlmc_ctx* ctx);
 

@@ -115,7 +115,8 @@ void run_band_norms(Workspace& ws, const void* g, int dtype, int64_t d, int M, i
 extern "C" {
 
 int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max) {
-    if (!out || d_max < 1 || d_max >= (int64_t(1) << 32) || M_max < 1 || L_max < 1 || L_max > kMaxLevels)
+    if (!out || d_max < 1 || d_max >= (int64_t(1) << 32) || M_max < 1 || M_max > kEmitMaxWorkers || L_max < 1 ||
+        L_max > kMaxLevels)
         return MLMC_ERR_ARG;
     DeviceGuard guard(device);
     if (!guard.ok) return MLMC_ERR_CUDA;

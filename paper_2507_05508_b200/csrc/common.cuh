@@ -16,9 +16,10 @@ constexpr uint32_t kKeyNone = 0xFFFFFFFFu;    // threshold above every finite ke
 constexpr uint32_t kNoSlot = 0xFFu;
 
 constexpr int kSweepThreads = 512;            // histogram / masked / norm sweeps
-constexpr int kEmitWorkers = 8;               // warps that count and write; one more warp per block computes the prefixes
-constexpr int kEmitThreads = (kEmitWorkers + 1) * 32;
+constexpr int kEmitWorkers = 8;               // warps that count and write; two more warps per block compute the prefixes
+constexpr int kEmitThreads = (kEmitWorkers + 2) * 32;
 constexpr int kEmitBlocksPerSM = 3;
+constexpr int kEmitMaxWorkers = 1024;         // M of one call: the emit kernel keeps every worker's band parameters in shared memory
 constexpr int kEmitRows = 16;                 // 32-bit words per lane per tile (1 fp32 or 2 bf16 elements each)
 constexpr int kEmitStages = 4;                // tiles of one block resident in shared memory
 constexpr int kEmitTile = kEmitWorkers * 32 * kEmitRows;   // words per tile = elements per fp32 tile; bf16: twice as many

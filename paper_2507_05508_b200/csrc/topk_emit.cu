@@ -19,7 +19,7 @@ namespace {
 
 constexpr unsigned kSpinLimit = 1u << 22;          // polls of a shared-memory word before a wait gives up
 constexpr unsigned kLookbackSpinLimit = 1u << 20;  // polls of a look-back record (each poll is a global load)
-constexpr int kTicketRing = 8;
+constexpr int kTicketRing = 16;
 
 // Look-back record of one tile: {C, A, B, state}: closed-range keys (Tb <= key <= Ta), keys equal to Ta,
 // keys equal to Tb; state 0 = not yet, 1 = the tile's own counts, 2 = running totals up to and including
@@ -94,7 +94,7 @@ struct EmitSync {
     unsigned tickets_ready;         // tickets [0, tickets_ready) of this block are in the ticket ring
     unsigned counted[kEmitStages];  // per slot: worker warps that have posted counts (kEmitWorkers more per tile;
                                     // per slot, because a fast warp may count tile k+1 before a slow one counts tile k)
-    unsigned prefix_ready;          // tiles [0, prefix_ready) of this block have their prefix in shared memory
+    unsigned ready[kEmitStages];    // per slot: j + 1 once tile j of this block has its prefix in shared memory
     int abort;                      // a bounded wait gave up: everybody leaves
 };
 
@@ -117,7 +117,6 @@ __device__ __forceinline__ bool wait_at_least(const unsigned* p, unsigned want, 
         }
     }
     ok = __all_sync(0xFFFFFFFFu, ok);
-    __threadfence_block();
     return ok;
 }
 
@@ -142,17 +141,26 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
     constexpr int kShare = kEmitRows * 32;
     extern __shared__ __align__(16) uint32_t sh_ring[];  // [kEmitStages][kEmitTile]
     __shared__ EmitSync sy;
-    __shared__ unsigned sh_ticket[kTicketRing];
-    __shared__ uint32_t sh_cC[kEmitStages][kEmitWorkers], sh_cA[kEmitStages][kEmitWorkers], sh_cB[kEmitStages][kEmitWorkers];
-    __shared__ uint32_t sh_wC[kEmitStages][kEmitWorkers], sh_wA[kEmitStages][kEmitWorkers], sh_wB[kEmitStages][kEmitWorkers];
-    __shared__ uint32_t sh_pre[kEmitStages][4];  // {C, A, B} before the tile; [3]: 1 = valid, 0 = skip the write
+    // The hand-over data is volatile and is published by a volatile flag store (or a shared-memory atomic) issued
+    // after it by the same thread: shared-memory accesses of one warp are performed in program order, so no fence
+    // is used (a fence would also wait for the asynchronous tile copies and the ticket atomic still in flight).
+    __shared__ volatile unsigned sh_ticket[kTicketRing];
+    // The counts of a tile are read by the workers when they write it, two iterations after counting; a fast warp
+    // may by then count the tile four ahead of a slow warp's write, so the counts keep eight tiles, not four.
+    constexpr int kCountSlots = 2 * kEmitStages;
+    __shared__ volatile uint32_t sh_cC[kCountSlots][kEmitWorkers], sh_cA[kCountSlots][kEmitWorkers], sh_cB[kCountSlots][kEmitWorkers];
+    __shared__ volatile uint32_t sh_pre[kEmitStages][4];  // {C, A, B} before the tile; [3]: 1 = valid, 0 = skip the write
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
     const unsigned kNone = 0xFFFFFFFFu;
+    // the band parameters of every worker, copied once (the ring is followed by M of them)
+    EmitParams* sh_emit = reinterpret_cast<EmitParams*>(sh_ring + kEmitStages * kEmitTile);
+    for (int i = threadIdx.x; i < M * (int)(sizeof(EmitParams) / 4); i += kEmitThreads)
+        reinterpret_cast<uint32_t*>(sh_emit)[i] = reinterpret_cast<const uint32_t*>(emit)[i];
 
     if (threadIdx.x == 0) {
-        sy.tickets_ready = 0; sy.prefix_ready = 0; sy.abort = 0;
-        for (int i = 0; i < kEmitStages; ++i) sy.counted[i] = 0;
+        sy.tickets_ready = 0; sy.abort = 0;
+        for (int i = 0; i < kEmitStages; ++i) sy.counted[i] = sy.ready[i] = 0;
     }
     __syncthreads();
 
@@ -162,7 +170,7 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
         auto fetch = [&](unsigned q, int k) {  // one commit per call, also for tiles that are skipped
             if (q < total_tiles) {
                 const int mq = (int)(q % (unsigned)M);
-                if (emit[mq].enabled)
+                if (sh_emit[mq].enabled)
                     emit_fetch_share<T>(g + (int64_t)mq * ld, d, (int64_t)(q / (unsigned)M),
                                         my_ring + (k & (kEmitStages - 1)) * kEmitTile, warp, lane);
             }
@@ -175,18 +183,41 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
         };
         unsigned q_m2 = kNone, q_m1 = kNone, q_0 = kNone, q_p1 = kNone;  // tiles k-2, k-1, k, k+1
         uint32_t fl_m2 = 0, fl_m1 = 0, ra_m2 = 0, ra_m1 = 0;              // their flags / row masks
+        // Worker warp 0 owns the tickets: one per iteration, for the tile three ahead, so every ticket is taken
+        // the same short time before its tile is counted and the tiles start in ticket order across the grid.
+        bool more = true;  // valid tickets may remain
+        auto put_ticket = [&](unsigned i, unsigned q) {
+            if (q >= total_tiles) {
+                q = kNone;
+                more = false;
+            }
+            if (lane == 0) {
+                sh_ticket[i & (kTicketRing - 1)] = q;
+                *reinterpret_cast<volatile unsigned*>(&sy.tickets_ready) = i + 1u;
+            }
+        };
+        if (warp == 0) {
+            unsigned base = 0;
+            if (lane == 0) base = atomicAdd(tile_counter, 3u);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            for (unsigned i = 0; i < 3u; ++i) put_ticket(i, base + i);
+        }
         bool alive = ticket_of(0, &q_0) && ticket_of(1, &q_p1);
         if (alive) {
             fetch(q_0, 0);
             fetch(q_p1, 1);
         }
         for (int k = 0; alive && (q_0 < total_tiles || q_m2 < total_tiles || q_m1 < total_tiles); ++k) {
+            // the ticket of tile k+3 is asked for now and handed out at the end of the iteration
+            unsigned q_new = kNone;
+            if (warp == 0 && more && lane == 0) q_new = atomicAdd(tile_counter, 1u);
+
             // ---- count this warp's share of tile k.
             // flags: bit i (fp32) or bits i and 16 + i (bf16 low / high half) = word i holds a closed-range key
             uint32_t flags = 0, rowany = 0;
             if (q_0 < total_tiles) {
                 const int mc_ = (int)(q_0 % (unsigned)M);
-                const EmitParams ec = emit[mc_];
+                const EmitParams ec = sh_emit[mc_];
                 uint32_t cC = 0, cA = 0, cB = 0;
                 cp_async_wait<1>();  // the share of tile k has landed (tile k+1 may still be in flight)
                 __syncwarp();
@@ -234,20 +265,31 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
                         cA = totCA >> 16;
                     }
                 }
+                // post the counts; the warp that posts last publishes the tile's record at once
+                const int cs = k & (kCountSlots - 1);
+                unsigned last = 0;
                 if (lane == 0) {
-                    const int slot = k & (kEmitStages - 1);
-                    sh_cC[slot][warp] = cC; sh_cA[slot][warp] = cA; sh_cB[slot][warp] = cB;
-                    __threadfence_block();
-                    atomicAdd(&sy.counted[slot], 1u);
+                    sh_cC[cs][warp] = cC; sh_cA[cs][warp] = cA; sh_cB[cs][warp] = cB;
+                    last = (atomicAdd(&sy.counted[k & (kEmitStages - 1)], 1u) + 1u ==
+                            ((unsigned)k / kEmitStages + 1u) * kEmitWorkers) ? 1u : 0u;
+                }
+                if (__shfl_sync(0xFFFFFFFFu, last, 0) && ec.enabled) {
+                    const uint32_t aggC = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cC[cs][lane] : 0u);
+                    const uint32_t aggA = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cA[cs][lane] : 0u);
+                    const uint32_t aggB = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cB[cs][lane] : 0u);
+                    const int tc = (int)(q_0 / (unsigned)M);
+                    // a worker's first tile has nothing before it: its counts are already running totals
+                    if (lane == 0)
+                        put_record(&tile_desc[(int64_t)mc_ * tiles_per_worker + tc], aggC, aggA, aggB, tc == 0 ? 2u : 1u);
                 }
             }
 
             // ---- write this warp's share of tile k-2
             if (q_m2 < total_tiles) {
                 const int mp = (int)(q_m2 % (unsigned)M), tp = (int)(q_m2 / (unsigned)M);
-                const EmitParams ep = emit[mp];
+                const EmitParams ep = sh_emit[mp];
                 const int slot = (k - 2) & (kEmitStages - 1);
-                if (!wait_at_least(&sy.prefix_ready, (unsigned)(k - 2) + 1u, &sy.abort)) {
+                if (!wait_at_least(&sy.ready[slot], (unsigned)(k - 2) + 1u, &sy.abort)) {
                     alive = false;
                     break;
                 }
@@ -255,10 +297,15 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
                     const uint32_t* tile = my_ring + slot * kEmitTile + lane;
                     const uint32_t Tb = min(ep.Tb, EW::kCap);
                     const uint32_t W = min(ep.Ta, EW::kCap) - Tb;
-                    uint32_t rA = sh_pre[slot][1] + sh_wA[slot][warp], rB = sh_pre[slot][2] + sh_wB[slot][warp];
-                    uint32_t base = band_prefix(sh_pre[slot][0] + sh_wC[slot][warp], rA, rB, ep.ra, ep.rb);
+                    // counts of the warps before this one in the tile (every warp of the tile has posted: the prefix is out)
+                    const int cs = (k - 2) & (kCountSlots - 1);
+                    const uint32_t wC = __reduce_add_sync(0xFFFFFFFFu, (lane < warp) ? sh_cC[cs][lane] : 0u);
+                    const uint32_t wA = __reduce_add_sync(0xFFFFFFFFu, (lane < warp) ? sh_cA[cs][lane] : 0u);
+                    const uint32_t wB = __reduce_add_sync(0xFFFFFFFFu, (lane < warp) ? sh_cB[cs][lane] : 0u);
+                    uint32_t rA = sh_pre[slot][1] + wA, rB = sh_pre[slot][2] + wB;
+                    uint32_t base = band_prefix(sh_pre[slot][0] + wC, rA, rB, ep.ra, ep.rb);
                     // ties in this warp's share?  (warp-uniform; ties elsewhere only move the base)
-                    const bool ties = (sh_cA[slot][warp] | sh_cB[slot][warp]) != 0u;
+                    const bool ties = (sh_cA[cs][warp] | sh_cB[cs][warp]) != 0u;
                     const float inv_p = (float)ep.inv_p;
                     uint32_t* idx_w = idx_out + (int64_t)mp * capacity;
                     float* val_w = val_out + (int64_t)mp * capacity;
@@ -323,6 +370,8 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
                 }
             }
 
+            if (warp == 0) put_ticket((unsigned)k + 3u, __shfl_sync(0xFFFFFFFFu, q_new, 0));
+
             // ---- start the copy of tile k+2 into the slot that tile k-2 has just left
             unsigned q_p2 = kNone;
             if (!ticket_of(k + 2, &q_p2)) {
@@ -337,84 +386,42 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
         }
         cp_async_wait<0>();
     } else {
-        // =========================== prefix warp ===========================
-        bool more = true;  // valid tickets may remain
-        auto put_ticket = [&](unsigned i, unsigned q) {
-            if (lane == 0) {
-                sh_ticket[i & (kTicketRing - 1)] = q;
-                __threadfence_block();
-                *reinterpret_cast<volatile unsigned*>(&sy.tickets_ready) = i + 1u;
-            }
-        };
-        auto take_ticket = [&]() -> unsigned {
-            unsigned q = kNone;
-            if (more && lane == 0) q = atomicAdd(tile_counter, 1u);
-            return q;
-        };
-        constexpr unsigned kAhead = 5;  // tickets kept ahead of the tile being handled (workers ask for tile k+2)
-        for (unsigned i = 0; i < kAhead; ++i) {
-            const unsigned q = __shfl_sync(0xFFFFFFFFu, take_ticket(), 0);
-            if (q >= total_tiles) more = false;
-            put_ticket(i, q);
-        }
-        // Tile j's counts are published as soon as its shares are counted; its look-back runs one tile later,
-        // while the workers count tile j+1.  By then the tiles that were counted at the same time as tile j
-        // have published their counts too, so the look-back does not wait for stragglers, and the nearest
-        // running total is about two rounds of the grid back: the window is 128 records wide.
-        constexpr int kWin = 4;  // records per lane and step
-        unsigned q_prev = kNone;
-        uint32_t aggC_p = 0, aggA_p = 0, aggB_p = 0;
-        for (unsigned j = 0;; ++j) {
-            // ask for the next ticket now, hand it out at the end of this tile: the atomic's latency stays hidden
-            const unsigned q_ahead = take_ticket();
-            const unsigned q = sh_ticket[j & (kTicketRing - 1)];
-            const bool cur_ok = q < total_tiles, prev_ok = q_prev < total_tiles;
-            if (!cur_ok && !prev_ok) break;  // tickets only grow: nothing valid follows (the tickets ahead are already out)
-            const int m = cur_ok ? (int)(q % (unsigned)M) : 0, t = cur_ok ? (int)(q / (unsigned)M) : 0;
-            const int mp = prev_ok ? (int)(q_prev % (unsigned)M) : 0, tp = prev_ok ? (int)(q_prev / (unsigned)M) : 0;
-            const EmitParams e = emit[m], ep = emit[mp];
-            const bool do_cur = cur_ok && e.enabled, do_prev = prev_ok && ep.enabled;
-            const int slot = j & (kEmitStages - 1), slot_p = (j - 1u) & (kEmitStages - 1);
-            uint4* desc = tile_desc + (int64_t)m * tiles_per_worker;
-            uint4* desc_p = tile_desc + (int64_t)mp * tiles_per_worker;
-            // first window of tile j-1's look-back: the loads fly while the workers count tile j.
-            // Lane i holds tiles look - i - 32 w, w = 0..3; positions before the worker's first tile are an empty total.
-            uint4 rec[kWin];
+        // =========================== prefix warps ===========================
+        // Two warps share the tiles of the block: warp pw handles tiles pw, pw + 2, ...  A tile's counts are
+        // published by the worker warp that posts last (nothing delays them); a prefix warp looks back for
+        // tile j once the block's next tile j+1 is counted too: by then the tiles that were counted at about
+        // the same time as tile j have published their counts, and the tiles one round of the grid earlier
+        // have their running totals, so the nearest running total lies inside the 128-record window.
+        const int pw = warp - kEmitWorkers;
+        constexpr int kWin = 4;  // look-back records per lane and step
+        for (unsigned j = (unsigned)pw;; j += 2) {
+            if (!wait_at_least(&sy.tickets_ready, j + 2u, &sy.abort)) break;  // tickets j and j+1 are out
+            const unsigned q = sh_ticket[j & (kTicketRing - 1)], q_next = sh_ticket[(j + 1u) & (kTicketRing - 1)];
+            if (q >= total_tiles) break;  // tickets only grow: nothing valid follows
+            const int m = (int)(q % (unsigned)M), t = (int)(q / (unsigned)M);
+            const int slot = (int)(j & (kEmitStages - 1));
+            if (!wait_at_least(&sy.counted[slot], (j / kEmitStages + 1u) * kEmitWorkers, &sy.abort)) break;
+            if (q_next < total_tiles &&
+                !wait_at_least(&sy.counted[(j + 1u) & (kEmitStages - 1)], ((j + 1u) / kEmitStages + 1u) * kEmitWorkers, &sy.abort))
+                break;
+            const EmitParams& e = sh_emit[m];
+            uint32_t pC = 0, pA = 0, pB = 0;
+            bool ok = true;
+            if (e.enabled) {
+                uint4* desc = tile_desc + (int64_t)m * tiles_per_worker;
+                const int cs = (int)(j & (kCountSlots - 1));
+                const uint32_t aggC = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cC[cs][lane] : 0u);
+                const uint32_t aggA = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cA[cs][lane] : 0u);
+                const uint32_t aggB = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cB[cs][lane] : 0u);
+                if (t > 0) {
+                    // lane i holds tiles look - i - 32 w; positions before the worker's first tile are an empty running total
+                    uint4 rec[kWin];
+                    int look = t - 1;
 #pragma unroll
-            for (int w = 0; w < kWin; ++w) {
-                const int at = tp - 1 - lane - 32 * w;
-                rec[w] = (do_prev && at >= 0) ? __ldcg(&desc_p[at]) : make_uint4(0u, 0u, 0u, 2u);
-            }
-            uint32_t aggC = 0, aggA = 0, aggB = 0;
-            if (cur_ok) {
-                if (!wait_at_least(&sy.counted[slot], (j / kEmitStages + 1u) * kEmitWorkers, &sy.abort)) break;
-                if (do_cur) {
-                    const uint32_t xC = (lane < kEmitWorkers) ? sh_cC[slot][lane] : 0u, xA = (lane < kEmitWorkers) ? sh_cA[slot][lane] : 0u,
-                                   xB = (lane < kEmitWorkers) ? sh_cB[slot][lane] : 0u;
-                    uint32_t iC = xC, iA = xA, iB = xB;
-#pragma unroll
-                    for (int o = 1; o < kEmitWorkers; o <<= 1) {
-                        const uint32_t yC = __shfl_up_sync(0xFFFFFFFFu, iC, o), yA = __shfl_up_sync(0xFFFFFFFFu, iA, o),
-                                       yB = __shfl_up_sync(0xFFFFFFFFu, iB, o);
-                        if (lane >= o) { iC += yC; iA += yA; iB += yB; }
+                    for (int w = 0; w < kWin; ++w) {
+                        const int at = look - lane - 32 * w;
+                        rec[w] = (at >= 0) ? __ldcg(&desc[at]) : make_uint4(0u, 0u, 0u, 2u);
                     }
-                    if (lane < kEmitWorkers) {
-                        sh_wC[slot][lane] = iC - xC;
-                        sh_wA[slot][lane] = iA - xA;
-                        sh_wB[slot][lane] = iB - xB;
-                    }
-                    aggC = __shfl_sync(0xFFFFFFFFu, iC, kEmitWorkers - 1);
-                    aggA = __shfl_sync(0xFFFFFFFFu, iA, kEmitWorkers - 1);
-                    aggB = __shfl_sync(0xFFFFFFFFu, iB, kEmitWorkers - 1);
-                    // a worker's first tile has nothing before it: its counts are already running totals
-                    if (lane == 0) put_record(&desc[t], aggC, aggA, aggB, t == 0 ? 2u : 1u);
-                }
-            }
-            if (prev_ok) {
-                uint32_t pC = 0, pA = 0, pB = 0;
-                bool ok = true;
-                if (do_prev && tp > 0) {
-                    int look = tp - 1;
                     unsigned spins = 0;
                     while (true) {
                         // nearest tile with a running total: everything nearer contributes its own counts,
@@ -434,7 +441,7 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
 #pragma unroll
                             for (int w = 0; w < kWin; ++w) {
                                 const int at = look - lane - 32 * w;
-                                if (at >= 0 && rec[w].w == 0u) rec[w] = __ldcg(&desc_p[at]);
+                                if (at >= 0 && rec[w].w == 0u) rec[w] = __ldcg(&desc[at]);
                             }
                             const bool bail = (++spins > kLookbackSpinLimit) || *reinterpret_cast<volatile int*>(&sy.abort) ||
                                               (*reinterpret_cast<volatile int*>(status) == MLMC_ERR_TIMEOUT);
@@ -462,31 +469,25 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
 #pragma unroll
                         for (int w = 0; w < kWin; ++w) {
                             const int at = look - lane - 32 * w;
-                            rec[w] = (at >= 0) ? __ldcg(&desc_p[at]) : make_uint4(0u, 0u, 0u, 2u);
+                            rec[w] = (at >= 0) ? __ldcg(&desc[at]) : make_uint4(0u, 0u, 0u, 2u);
                         }
                     }
-                    if (lane == 0) put_record(&desc_p[tp], pC + aggC_p, pA + aggA_p, pB + aggB_p, 2u);  // also after a give-up
+                    if (lane == 0) put_record(&desc[t], pC + aggC, pA + aggA, pB + aggB, 2u);  // also after a give-up
                     if (!ok) {
                         set_status(status, MLMC_ERR_TIMEOUT);
-                        worker_err[mp] = MLMC_ERR_TIMEOUT;
+                        worker_err[m] = MLMC_ERR_TIMEOUT;
                     }
                 }
                 // self-check on the worker's last tile: the band has exactly k_l - k_{l-1} entries
-                if (lane == 0 && do_prev && ok && tp == tiles_per_worker - 1 &&
-                    band_prefix(pC + aggC_p, pA + aggA_p, pB + aggB_p, ep.ra, ep.rb) != ep.expect)
+                if (lane == 0 && ok && t == tiles_per_worker - 1 &&
+                    band_prefix(pC + aggC, pA + aggA, pB + aggB, e.ra, e.rb) != e.expect)
                     set_status(status, MLMC_ERR_INTERNAL);
-                if (lane == 0) {
-                    sh_pre[slot_p][0] = pC; sh_pre[slot_p][1] = pA; sh_pre[slot_p][2] = pB;
-                    sh_pre[slot_p][3] = (do_prev && ok) ? 1u : 0u;
-                    __threadfence_block();
-                    *reinterpret_cast<volatile unsigned*>(&sy.prefix_ready) = j;  // tiles [0, j) have their prefix
-                }
             }
-            const unsigned qa = __shfl_sync(0xFFFFFFFFu, q_ahead, 0);
-            if (qa >= total_tiles) more = false;
-            put_ticket(j + kAhead, qa);
-            q_prev = q;
-            aggC_p = aggC; aggA_p = aggA; aggB_p = aggB;
+            if (lane == 0) {
+                sh_pre[slot][0] = pC; sh_pre[slot][1] = pA; sh_pre[slot][2] = pB;
+                sh_pre[slot][3] = (e.enabled && ok) ? 1u : 0u;
+                *reinterpret_cast<volatile unsigned*>(&sy.ready[slot]) = j + 1u;
+            }
         }
     }
     if (*reinterpret_cast<volatile int*>(&sy.abort)) set_status(status, MLMC_ERR_TIMEOUT);
@@ -525,8 +526,10 @@ aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict_
             if (o1 > o0) {
                 const uint32_t* a = idx + (int64_t)m * capacity;
                 const float* v = val + (int64_t)m * capacity;
-                for (uint32_t j = o0 + threadIdx.x; j < o1; j += blockDim.x)
-                    acc[a[j] - (uint32_t)base] += v[j];  // indices are unique within a worker
+                for (uint32_t j = o0 + threadIdx.x; j < o1; j += blockDim.x) {
+                    const uint32_t off = a[j] - (uint32_t)base;  // indices are unique within a worker
+                    if (off < (uint32_t)kAggTile) acc[off] += v[j];  // a message that is not index-sorted cannot reach outside the tile
+                }
                 __syncthreads();
             }
         }
@@ -539,7 +542,7 @@ aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict_
 }  // namespace
 
 int configure_emit_kernels() {
-    const int smem = kEmitStages * kEmitTile * (int)sizeof(uint32_t);
+    const int smem = kEmitStages * kEmitTile * (int)sizeof(uint32_t) + kEmitMaxWorkers * (int)sizeof(EmitParams);  // ring + band parameters
     if (cudaFuncSetAttribute(emit_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return MLMC_ERR_CUDA;
     if (cudaFuncSetAttribute(emit_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
@@ -557,7 +560,7 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
     cudaMemsetAsync(ws.tile_counter, 0, sizeof(unsigned), s);
     unsigned grid = (unsigned)(ws.sm_count * kEmitBlocksPerSM);  // persistent blocks
     if (grid > total) grid = total;
-    const size_t smem = (size_t)kEmitStages * kEmitTile * sizeof(uint32_t);
+    const size_t smem = (size_t)kEmitStages * kEmitTile * sizeof(uint32_t) + (size_t)M * sizeof(EmitParams);
     LaunchScope t(ws, K_EMIT, s);
     if (dtype == MLMC_BF16)
         emit_kernel<bf16_t><<<grid, kEmitThreads, smem, s>>>(static_cast<const bf16_t*>(g), d, ld, tpw, total, M, ws.emit,
