@@ -115,6 +115,7 @@ __device__ __forceinline__ bool wait_at_least(const unsigned* p, unsigned want, 
             ok = false;
             break;
         }
+        __nanosleep(64);  // a waiting warp leaves the issue slots to the warps that have work
     }
     ok = __all_sync(0xFFFFFFFFu, ok);
     return ok;
@@ -144,7 +145,8 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
     // The hand-over data is volatile and is published by a volatile flag store (or a shared-memory atomic) issued
     // after it by the same thread: shared-memory accesses of one warp are performed in program order, so no fence
     // is used (a fence would also wait for the asynchronous tile copies and the ticket atomic still in flight).
-    __shared__ volatile unsigned sh_ticket[kTicketRing];
+    __shared__ volatile unsigned sh_ticket[kTicketRing];          // tile k of this block: its ticket q ...
+    __shared__ volatile int sh_tm[kTicketRing], sh_tt[kTicketRing];  // ... its worker q % M and its tile index q / M
     // The counts of a tile are read by the workers when they write it, two iterations after counting; a fast warp
     // may by then count the tile four ahead of a slow warp's write, so the counts keep eight tiles, not four.
     constexpr int kCountSlots = 2 * kEmitStages;
@@ -169,9 +171,9 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
         uint32_t* my_ring = sh_ring + warp * kShare;
         auto fetch = [&](unsigned q, int k) {  // one commit per call, also for tiles that are skipped
             if (q < total_tiles) {
-                const int mq = (int)(q % (unsigned)M);
+                const int mq = sh_tm[k & (kTicketRing - 1)];
                 if (sh_emit[mq].enabled)
-                    emit_fetch_share<T>(g + (int64_t)mq * ld, d, (int64_t)(q / (unsigned)M),
+                    emit_fetch_share<T>(g + (int64_t)mq * ld, d, (int64_t)sh_tt[k & (kTicketRing - 1)],
                                         my_ring + (k & (kEmitStages - 1)) * kEmitTile, warp, lane);
             }
             cp_async_commit();
@@ -192,6 +194,8 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
                 more = false;
             }
             if (lane == 0) {
+                sh_tm[i & (kTicketRing - 1)] = (int)(q % (unsigned)M);  // divided once here, read by every warp
+                sh_tt[i & (kTicketRing - 1)] = (int)(q / (unsigned)M);
                 sh_ticket[i & (kTicketRing - 1)] = q;
                 *reinterpret_cast<volatile unsigned*>(&sy.tickets_ready) = i + 1u;
             }
@@ -216,7 +220,7 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
             // flags: bit i (fp32) or bits i and 16 + i (bf16 low / high half) = word i holds a closed-range key
             uint32_t flags = 0, rowany = 0;
             if (q_0 < total_tiles) {
-                const int mc_ = (int)(q_0 % (unsigned)M);
+                const int mc_ = sh_tm[k & (kTicketRing - 1)];
                 const EmitParams ec = sh_emit[mc_];
                 uint32_t cC = 0, cA = 0, cB = 0;
                 cp_async_wait<1>();  // the share of tile k has landed (tile k+1 may still be in flight)
@@ -277,7 +281,7 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
                     const uint32_t aggC = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cC[cs][lane] : 0u);
                     const uint32_t aggA = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cA[cs][lane] : 0u);
                     const uint32_t aggB = __reduce_add_sync(0xFFFFFFFFu, (lane < kEmitWorkers) ? sh_cB[cs][lane] : 0u);
-                    const int tc = (int)(q_0 / (unsigned)M);
+                    const int tc = sh_tt[k & (kTicketRing - 1)];
                     // a worker's first tile has nothing before it: its counts are already running totals
                     if (lane == 0)
                         put_record(&tile_desc[(int64_t)mc_ * tiles_per_worker + tc], aggC, aggA, aggB, tc == 0 ? 2u : 1u);
@@ -286,7 +290,7 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
 
             // ---- write this warp's share of tile k-2
             if (q_m2 < total_tiles) {
-                const int mp = (int)(q_m2 % (unsigned)M), tp = (int)(q_m2 / (unsigned)M);
+                const int mp = sh_tm[(k - 2) & (kTicketRing - 1)], tp = sh_tt[(k - 2) & (kTicketRing - 1)];
                 const EmitParams ep = sh_emit[mp];
                 const int slot = (k - 2) & (kEmitStages - 1);
                 if (!wait_at_least(&sy.ready[slot], (unsigned)(k - 2) + 1u, &sy.abort)) {
@@ -398,7 +402,7 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
             if (!wait_at_least(&sy.tickets_ready, j + 2u, &sy.abort)) break;  // tickets j and j+1 are out
             const unsigned q = sh_ticket[j & (kTicketRing - 1)], q_next = sh_ticket[(j + 1u) & (kTicketRing - 1)];
             if (q >= total_tiles) break;  // tickets only grow: nothing valid follows
-            const int m = (int)(q % (unsigned)M), t = (int)(q / (unsigned)M);
+            const int m = sh_tm[j & (kTicketRing - 1)], t = sh_tt[j & (kTicketRing - 1)];
             const int slot = (int)(j & (kEmitStages - 1));
             if (!wait_at_least(&sy.counted[slot], (j / kEmitStages + 1u) * kEmitWorkers, &sy.abort)) break;
             if (q_next < total_tiles &&
