@@ -515,19 +515,23 @@ __global__ void agg_offsets_kernel(const uint32_t* __restrict__ idx, const int64
     offsets[i] = (uint32_t)lo;
 }
 
+// M is at most kEmitMaxWorkers: the offsets of all workers for one tile are fetched together.
 __global__ void __launch_bounds__(256)
 aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict__ val, int64_t capacity, int M,
                       int64_t d, int ntiles, const uint32_t* __restrict__ offsets, float* __restrict__ out) {
-    __shared__ float acc[kAggTile];
-    const float fM = (float)M;
+    __shared__ __align__(16) float acc[kAggTile];
+    extern __shared__ uint32_t sh_off[];  // [2 M]: first and one-past-last message entry of every worker in this tile
+    const float inv_M = 1.0f / (float)M;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
         const int64_t base = (int64_t)t * kAggTile;
-        for (int i = threadIdx.x; i < kAggTile; i += blockDim.x) acc[i] = 0.0f;
+        for (int i = threadIdx.x; i < 2 * M; i += blockDim.x)
+            sh_off[i] = offsets[(int64_t)(i >> 1) * (ntiles + 1) + t + (i & 1)];
+        for (int i = threadIdx.x; i < kAggTile / 4; i += blockDim.x)
+            reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         __syncthreads();
         for (int m = 0; m < M; ++m) {  // fixed worker order: reproducible fp32 sums
-            const uint32_t o0 = offsets[(int64_t)m * (ntiles + 1) + t];
-            const uint32_t o1 = offsets[(int64_t)m * (ntiles + 1) + t + 1];
-            if (o1 > o0) {
+            const uint32_t o0 = sh_off[2 * m], o1 = sh_off[2 * m + 1];
+            if (o1 > o0) {  // block-uniform
                 const uint32_t* a = idx + (int64_t)m * capacity;
                 const float* v = val + (int64_t)m * capacity;
                 for (uint32_t j = o0 + threadIdx.x; j < o1; j += blockDim.x) {
@@ -537,8 +541,16 @@ aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict_
                 __syncthreads();
             }
         }
-        for (int i = threadIdx.x; i < kAggTile; i += blockDim.x)
-            if (base + i < d) out[base + i] = acc[i] / fM;
+        if (base + kAggTile <= d && (d & 3) == 0) {
+            for (int i = threadIdx.x; i < kAggTile / 4; i += blockDim.x) {
+                float4 x = reinterpret_cast<const float4*>(acc)[i];
+                x.x *= inv_M; x.y *= inv_M; x.z *= inv_M; x.w *= inv_M;
+                reinterpret_cast<float4*>(out + base)[i] = x;
+            }
+        } else {
+            for (int i = threadIdx.x; i < kAggTile; i += blockDim.x)
+                if (base + i < d) out[base + i] = acc[i] * inv_M;
+        }
         __syncthreads();
     }
 }
@@ -587,7 +599,8 @@ void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int
     int grid = ws.sm_count * 8;
     if (grid > ntiles) grid = ntiles;
     LaunchScope t(ws, K_AGG_TOPK, s);
-    aggregate_topk_kernel<<<grid, 256, 0, s>>>(msgs.idx, msgs.val, msgs.capacity, M, d, ntiles, ws.agg_offsets, out);
+    aggregate_topk_kernel<<<grid, 256, 2 * M * sizeof(uint32_t), s>>>(msgs.idx, msgs.val, msgs.capacity, M, d, ntiles,
+                                                                      ws.agg_offsets, out);
 }
 
 }  // namespace mlmc
@@ -614,7 +627,7 @@ int g_static_sm_count[kMaxDevices];
 extern "C" int mlmc_aggregate_topk_noalloc(const mlmc_topk_msgs* msgs, int M, int64_t d, float* out, void* stream) {
     using namespace mlmc;
     if (!msgs || !out || !msgs->idx || !msgs->val || !msgs->count || !msgs->level) return MLMC_ERR_ARG;
-    if (M < 1 || d < 1 || d >= (int64_t(1) << 32) || msgs->capacity < 0) return MLMC_ERR_ARG;
+    if (M < 1 || M > kEmitMaxWorkers || d < 1 || d >= (int64_t(1) << 32) || msgs->capacity < 0) return MLMC_ERR_ARG;
     const int64_t ntiles = (d + kAggTile - 1) / kAggTile;
     const int64_t n_off = (int64_t)M * (ntiles + 1);
     if (n_off > kStaticOffsetWords) return MLMC_ERR_ARG;  // beyond the fixed scratch: use mlmc_aggregate with a context
@@ -641,7 +654,7 @@ extern "C" int mlmc_aggregate_topk_noalloc(const mlmc_topk_msgs* msgs, int M, in
                                                                        msgs->capacity, M, (int)ntiles, offsets);
     int64_t grid = (int64_t)g_static_sm_count[dev] * 8;
     if (grid > ntiles) grid = ntiles;
-    aggregate_topk_kernel<<<(unsigned)grid, 256, 0, s>>>(msgs->idx, msgs->val, msgs->capacity, M, d, (int)ntiles,
-                                                         offsets, out);
+    aggregate_topk_kernel<<<(unsigned)grid, 256, 2 * M * sizeof(uint32_t), s>>>(msgs->idx, msgs->val, msgs->capacity, M, d,
+                                                                                (int)ntiles, offsets, out);
     return cudaGetLastError() == cudaSuccess ? MLMC_OK : MLMC_ERR_CUDA;
 }
