@@ -32,7 +32,11 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic per launch of each sweep kernel relative to its algorithmic bytes, from the ncu captures
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same
 # kernel; traffic grows in proportion to the elements swept).  None = not captured yet.
-NCU_TRAFFIC_RATIO = {}
+NCU_TRAFFIC_RATIO = {
+    # profiles/c5_small_kernels.md (fp32, d = 32e6, M = 4)
+    "hist1:f32": 1.007, "sums_candidates:f32": 1.011, "emit:f32": 1.00, "absmax:f32": 1.008, "bit_stats:f32": 1.009,
+    "bit_pack:f32": 1.00,
+}
 
 
 def parse_args():
