@@ -252,11 +252,17 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
 #pragma unroll
                         for (int i = 0; i < kEmitRows; ++i) {
                             const uint32_t k2 = tile[i * 32] & 0x7FFF7FFFu;
-                            const uint32_t f = (k2 + geB) & (leA - k2) & hi;
-                            flags |= f >> (15 - i);
-                            const uint32_t fB = f & ~(k2 + geB1);
-                            const uint32_t fA = f & ~((leA1 - k2) & keepA1);
-                            acc += (fA >> 15) + (fB >> 7);  // 5-bit counters: A at bits 0 / 16, B at bits 8 / 24
+                            flags |= ((k2 + geB) & (leA - k2) & hi) >> (15 - i);
+                        }
+                        if (__any_sync(0xFFFFFFFFu, flags != 0u)) {  // ties are closed-range keys: look only if there are any
+#pragma unroll
+                            for (int i = 0; i < kEmitRows; ++i) {
+                                const uint32_t k2 = tile[i * 32] & 0x7FFF7FFFu;
+                                const uint32_t f = (k2 + geB) & (leA - k2) & hi;
+                                const uint32_t fB = f & ~(k2 + geB1);
+                                const uint32_t fA = f & ~((leA1 - k2) & keepA1);
+                                acc += (fA >> 15) + (fB >> 7);  // 5-bit counters: A at bits 0 / 16, B at bits 8 / 24
+                            }
                         }
                         cA = (acc & 0x1Fu) + ((acc >> 16) & 0x1Fu);
                         cB = ((acc >> 8) & 0x1Fu) + ((acc >> 24) & 0x1Fu);
@@ -309,7 +315,16 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
                     uint32_t rA = sh_pre[slot][1] + wA, rB = sh_pre[slot][2] + wB;
                     uint32_t base = band_prefix(sh_pre[slot][0] + wC, rA, rB, ep.ra, ep.rb);
                     // ties in this warp's share?  (warp-uniform; ties elsewhere only move the base)
-                    const bool ties = (sh_cA[cs][warp] | sh_cB[cs][warp]) != 0u;
+                    // Ties in this warp's share (warp-uniform; ties elsewhere only move the base).  Unless the cut
+                    // rank of a threshold falls among this share's ties, all of them are on one side of it: the
+                    // ties of Ta all outside Top-k_{l-1} (in the band) or all inside (dropped), the ties of Tb all
+                    // inside Top-k_l (in the band) or all outside (dropped).  Only the share that holds a cut
+                    // ranks its ties one by one.
+                    const uint32_t myA = sh_cA[cs][warp], myB = sh_cB[cs][warp];
+                    const bool dropA = myA != 0u && rA + myA <= ep.ra, keepA = myA == 0u || rA >= ep.ra;
+                    const bool dropB = myB != 0u && rB >= ep.rb, keepB = myB == 0u || rB + myB <= ep.rb;
+                    const bool ties = !((keepA || dropA) && (keepB || dropB)) || ((myA | myB) != 0u && W == 0u);
+                    const bool drop_any = !ties && (dropA || dropB);
                     const float inv_p = (float)ep.inv_p;
                     uint32_t* idx_w = idx_out + (int64_t)mp * capacity;
                     float* val_w = val_out + (int64_t)mp * capacity;
@@ -328,6 +343,10 @@ emit_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker
 #pragma unroll
                             for (int s = 0; s < S; ++s) {
                                 em[s] = (fl_m2 >> (i + 16 * s)) & 1u;
+                                if (drop_any) {  // warp-uniform
+                                    const uint32_t tk = EW::key(w, s) - Tb;
+                                    em[s] = em[s] && !(dropA && tk == W) && !(dropB && tk == 0u);
+                                }
                                 me[s] = __ballot_sync(0xFFFFFFFFu, em[s]);
                             }
                         } else {
