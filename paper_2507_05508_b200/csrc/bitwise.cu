@@ -104,7 +104,10 @@ absmax_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* gmax_bit
 }
 
 // ---- adaptive only: exact field energies S_l = sum_i f_l^2 for every level in one sweep
-template <typename T, int LMAX>
+// Acc = uint32_t when every field is at most 8 bits wide and a thread sees fewer than 2^16 entries (f^2 < 2^16,
+// so the sum fits 32 bits), else unsigned long long.  Fields come from the prefix codes P_l = q >> (B - b_l):
+// f_l = P_l - (P_{l-1} << w_l), one shift and one multiply-add per level.
+template <typename T, int LMAX, typename Acc>
 __global__ void __launch_bounds__(kSweepThreads)
 bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* __restrict__ gmax_bits,
                  BitSchedule sc, unsigned long long* __restrict__ S_partial, int stat_ctas, const int* worker_err) {
@@ -114,14 +117,14 @@ bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t*
     if (worker_err[m]) return;
     const float gmax = __uint_as_float(gmax_bits[m]);
     const Quantiser qz(gmax, sc.B);
-    unsigned long long acc[LMAX];
+    Acc acc[LMAX];
     int sh[LMAX];
-    uint32_t mk[LMAX];
+    uint32_t neg_pow[LMAX];
 #pragma unroll
-    for (int l = 0; l < LMAX; ++l) {  // the schedule in registers; levels past L get an empty mask and add nothing
+    for (int l = 0; l < LMAX; ++l) {  // the schedule in registers; levels past L get shift 0 and width 0: their field is q - q = 0
         acc[l] = 0;
         sh[l] = (l < sc.L) ? sc.shift[l] : 0;
-        mk[l] = (l < sc.L) ? sc.mask[l] : 0u;
+        neg_pow[l] = 0u - (1u << ((l < sc.L) ? sc.width[l] : 0));
     }
     if (gmax > 0.0f) {
         const T* row = g + (int64_t)m * ld;
@@ -129,10 +132,13 @@ bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t*
         block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
         auto take = [&](uint32_t bits) {
             const uint32_t q = qz.code(__float_as_uint(Tr::value(bits)) & 0x7FFFFFFFu);
+            uint32_t prev = 0;  // P_{l-1}
 #pragma unroll
             for (int l = 0; l < LMAX; ++l) {
-                const uint32_t f = (q >> sh[l]) & mk[l];
-                acc[l] += (unsigned long long)f * f;
+                const uint32_t P = q >> sh[l];
+                const uint32_t f = prev * neg_pow[l] + P;
+                acc[l] += (Acc)f * f;
+                prev = P;
             }
         };
         // two 16-byte loads per thread are in flight before either is used
@@ -158,7 +164,7 @@ bit_stats_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t*
 #pragma unroll
     for (int l = 0; l < LMAX; ++l) {
         if (l >= sc.L) break;
-        unsigned long long x = acc[l];
+        unsigned long long x = (unsigned long long)acc[l];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
         if ((threadIdx.x & 31) == 0) sh_red[threadIdx.x >> 5] = x;
@@ -453,19 +459,19 @@ void launch_absmax(Workspace& ws, const void* g, int dtype, int64_t d, int M, in
     }
 }
 
-template <typename T>
+template <typename T, typename Acc>
 static void launch_bit_stats_t(Workspace& ws, const T* g, int64_t d, int M, int64_t ld, const BitSchedule& sc, int nb,
                                cudaStream_t s) {
     dim3 grid(nb, M);
-    if (sc.L <= 8)
-        bit_stats_kernel<T, 8><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas,
-                                                              ws.worker_err);
-    else if (sc.L <= 16)
-        bit_stats_kernel<T, 16><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas,
-                                                               ws.worker_err);
-    else
-        bit_stats_kernel<T, 23><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas,
-                                                               ws.worker_err);
+#define MLMC_BIT_STATS(LM)                                                                                          \
+    bit_stats_kernel<T, LM, Acc><<<grid, kSweepThreads, 0, s>>>(g, d, ld, ws.gmax_bits, sc, ws.S_partial, ws.stat_ctas, \
+                                                               ws.worker_err)
+    if (sc.L <= 4) MLMC_BIT_STATS(4);
+    else if (sc.L <= 6) MLMC_BIT_STATS(6);
+    else if (sc.L <= 8) MLMC_BIT_STATS(8);
+    else if (sc.L <= 16) MLMC_BIT_STATS(16);
+    else MLMC_BIT_STATS(23);
+#undef MLMC_BIT_STATS
 }
 
 void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
@@ -475,11 +481,21 @@ void launch_bit_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M,
     int nb = bit_blocks(ws, d, dtype == MLMC_BF16 ? 8 : 4, M, 4);
     if (nb > ws.stat_ctas) nb = ws.stat_ctas;
     ws.cur_stat_ctas = nb;
+    // 32-bit sums are exact while f^2 < 2^16 and a thread adds fewer than 2^16 of them
+    const int vec = dtype == MLMC_BF16 ? 8 : 4;
+    const int64_t vec_per_block = ((d + vec - 1) / vec + nb - 1) / nb;
+    const int64_t per_thread = ((vec_per_block + kSweepThreads - 1) / kSweepThreads + 1) * vec;
+    int w_top = 0;
+    for (int l = 0; l < L; ++l) w_top = sc.width[l] > w_top ? sc.width[l] : w_top;
+    const bool narrow = w_top <= 8 && per_thread < 65536;
     LaunchScope t(ws, K_BIT_STATS, s);
-    if (dtype == MLMC_BF16)
-        launch_bit_stats_t<bf16_t>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, nb, s);
-    else
-        launch_bit_stats_t<float>(ws, static_cast<const float*>(g), d, M, ld, sc, nb, s);
+    if (dtype == MLMC_BF16) {
+        if (narrow) launch_bit_stats_t<bf16_t, uint32_t>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, nb, s);
+        else launch_bit_stats_t<bf16_t, unsigned long long>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, nb, s);
+    } else {
+        if (narrow) launch_bit_stats_t<float, uint32_t>(ws, static_cast<const float*>(g), d, M, ld, sc, nb, s);
+        else launch_bit_stats_t<float, unsigned long long>(ws, static_cast<const float*>(g), d, M, ld, sc, nb, s);
+    }
 }
 
 void launch_bit_probs_draw(Workspace& ws, int M, const int32_t* b, int L, bool adaptive, bool need_delta,

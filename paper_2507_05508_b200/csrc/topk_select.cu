@@ -137,34 +137,6 @@ __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t x) {
     return x;
 }
 
-// Exclusive prefix over threads in DESCENDING thread order (thread t gets the sum of threads > t).
-__device__ uint32_t block_exclusive_suffix(uint32_t x, uint32_t* sh_warp /* [32] */) {
-    const int nt = blockDim.x;
-    const int rt = nt - 1 - threadIdx.x;  // reversed thread index
-    // emulate a forward scan over reversed indices by exchanging through shared memory
-    __shared__ uint32_t sh_x[kResolveThreads];
-    sh_x[rt] = x;
-    __syncthreads();
-    const uint32_t mine = sh_x[threadIdx.x];  // value of reversed position threadIdx.x
-    const uint32_t inc = warp_inclusive_sum(mine);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 31) sh_warp[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        const uint32_t w = (lane < (nt >> 5)) ? sh_warp[lane] : 0u;
-        const uint32_t winc = warp_inclusive_sum(w);
-        sh_warp[lane] = winc - w;
-    }
-    __syncthreads();
-    const uint32_t exc = inc - mine + sh_warp[warp];  // exclusive prefix at reversed position threadIdx.x
-    __syncthreads();
-    sh_x[threadIdx.x] = exc;
-    __syncthreads();
-    const uint32_t res = sh_x[rt];
-    __syncthreads();
-    return res;
-}
-
 // Assigns histogram slots to live queries: queries whose fixed prefix (>> shift) agree share a slot.
 __device__ void assign_slots(Query* q, int nq, int shift) {
     int next = 0;
@@ -192,14 +164,36 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is
     const int m = blockIdx.x;
     uint32_t* S = hist1 + (int64_t)m * kBins1;
     Query* q = queries + m * kMaxQueries;
-    constexpr int per = kBins1 / kResolveThreads;  // 32 bins per thread
-    const int b0 = threadIdx.x * per;
-    uint32_t local = 0;
-    for (int i = 0; i < per; ++i) local += S[b0 + i];
-    uint32_t above = block_exclusive_suffix(local, sh_warp);
-    for (int i = per - 1; i >= 0; --i) {
-        above += S[b0 + i];
-        S[b0 + i] = above;
+    constexpr int per = kBins1 / kResolveThreads;  // 32 chunks of 1024 bins; thread t owns bin c * 1024 + t of chunk c
+    {
+        // suffix sums S[b] = #{digit >= b}, chunk by chunk from the top, coalesced
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        uint32_t carry = 0;
+        uint32_t cnt[per];
+#pragma unroll
+        for (int c = 0; c < per; ++c) cnt[c] = S[c * kResolveThreads + threadIdx.x];  // all 32 loads in flight at once
+#pragma unroll
+        for (int c = per - 1; c >= 0; --c) {
+            const int b = c * kResolveThreads + threadIdx.x;
+            uint32_t v = cnt[c];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {  // inclusive suffix within the warp
+                const uint32_t y = __shfl_down_sync(0xFFFFFFFFu, v, o);
+                if (lane + o < 32) v += y;
+            }
+            if (lane == 0) sh_warp[warp] = v;
+            __syncthreads();
+            uint32_t higher = 0, total = 0;
+#pragma unroll 8
+            for (int w = 0; w < kResolveThreads / 32; ++w) {
+                const uint32_t x = sh_warp[w];
+                total += x;
+                if (w > warp) higher += x;
+            }
+            S[b] = v + higher + carry;
+            carry += total;
+            __syncthreads();
+        }
     }
     __syncthreads();
     if (worker_err[m]) return;
@@ -234,7 +228,7 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is
     __syncthreads();
     uint8_t* tab = table1 + (int64_t)m * kBins1;
     for (int i = 0; i < per; ++i) {
-        const int b = b0 + i;
+        const int b = i * kResolveThreads + threadIdx.x;
         uint32_t code = 0;
         for (int j = 0; j < nq; ++j) {
             if (sh_bin[j] > b) ++code;
@@ -641,7 +635,7 @@ norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query*
         const int64_t lo = (l == L - 1) ? -1 : (int64_t)sh_thr[l];
         double acc = 0.0;
         for (int i = 0; i < per; ++i) {
-            const uint32_t key = threadIdx.x * per + i;
+            const uint32_t key = i * kResolveThreads + threadIdx.x;  // coalesced over the block
             if ((int64_t)key > lo && key < hi) {
                 const uint32_t cnt = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
                 if (cnt) {  // empty bins include the Inf/NaN encodings, whose value must not enter the sum
