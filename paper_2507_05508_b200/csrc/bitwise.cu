@@ -270,7 +270,7 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
     using Tr = ElemTraits<T>;
     constexpr int kGroup = 1024;
     constexpr int kGroupBytes = kGroup * (int)sizeof(T);
-    extern __shared__ __align__(16) uint8_t sh_pack[];  // [warps][2][kGroupBytes]
+    extern __shared__ __align__(16) uint8_t sh_pack[];  // [warps][2][kGroupBytes], then [warps][1024] field bytes
     const int m = blockIdx.y;
     const int level = bit_level[m];
     if (level < 0) return;
@@ -285,6 +285,7 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
     const T* row = g + (int64_t)m * ld;
     uint32_t* out = planes + (int64_t)m * (1 + w_max) * words;
     uint8_t* ring = sh_pack + warp * 2 * kGroupBytes;
+    uint8_t* bytes = sh_pack + warps_per_block * 2 * kGroupBytes + warp * 1024;  // 32 rows x 32 field bytes
     auto fetch = [&](int64_t grp, int stage) {  // one commit per call
         if (grp < ngroups) {
             const int64_t e0 = grp * kGroup;
@@ -325,15 +326,41 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
             code[s] = ((q >> shift) & mask) | (__float_as_uint(x) & 0x80000000u);
         }
         const int64_t word = grp * 32 + lane;
-        for (int j = 0; j <= w; ++j) {
-            const int bit = (j == 0) ? 31 : (w - j);
-            uint32_t mine = 0;
+        if (w <= 8) {
+            // Fields of at most 8 bits go through a byte matrix in shared memory: lane L writes the field of each of
+            // its 32 rows, then lane r gathers bit b of the 32 bytes of row r, four bytes per multiply
+            // (((x >> b) & 0x01010101) * 0x01020408 puts the four bits side by side in bits 24..27).  This costs
+            // a quarter of one ballot per row and plane.  The sign plane takes one ballot per row.
+            uint32_t sign_w = 0;
 #pragma unroll
             for (int s = 0; s < 32; ++s) {
-                const uint32_t b = __ballot_sync(0xFFFFFFFFu, (code[s] >> bit) & 1u);
-                if (lane == s) mine = b;
+                const uint32_t bs = __ballot_sync(0xFFFFFFFFu, (int)code[s] < 0);
+                if (lane == s) sign_w = bs;
+                bytes[s * 32 + lane] = (uint8_t)code[s];
             }
-            if (word < words) out[(int64_t)j * words + word] = mine;
+            __syncwarp();
+            const uint4 lo = reinterpret_cast<const uint4*>(bytes + lane * 32)[0];
+            const uint4 hi = reinterpret_cast<const uint4*>(bytes + lane * 32)[1];
+            const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            if (word < words) out[word] = sign_w;
+            for (int j = 1; j <= w; ++j) {
+                const int bit = w - j;
+                uint32_t pw = 0;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) pw |= ((((x[c] >> bit) & 0x01010101u) * 0x01020408u) >> 24 & 0xFu) << (4 * c);
+                if (word < words) out[(int64_t)j * words + word] = pw;
+            }
+        } else {
+            for (int j = 0; j <= w; ++j) {
+                const int bit = (j == 0) ? 31 : (w - j);
+                uint32_t mine = 0;
+#pragma unroll
+                for (int s = 0; s < 32; ++s) {
+                    const uint32_t b = __ballot_sync(0xFFFFFFFFu, (code[s] >> bit) & 1u);
+                    if (lane == s) mine = b;
+                }
+                if (word < words) out[(int64_t)j * words + word] = mine;
+            }
         }
         __syncwarp();  // everyone is done with this slot before the copy after next lands in it
     }
@@ -440,7 +467,7 @@ int bit_blocks(const Workspace& ws, int64_t d, int vec, int M, int waves) {
 
 int configure_bit_kernels() {
     if (cudaFuncSetAttribute(bit_pack_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (kBitThreads / 32) * 2 * 1024 * 4) != cudaSuccess)
+                             (kBitThreads / 32) * (2 * 1024 * 4 + 1024)) != cudaSuccess)
         return MLMC_ERR_CUDA;
     return MLMC_OK;
 }
@@ -520,10 +547,10 @@ void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, 
     if (nb < 1) nb = 1;
     LaunchScope t(ws, K_BIT_PACK, s);
     if (dtype == MLMC_BF16)
-        bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * 2 * 1024 * 2, s>>>(
+        bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * (2 * 1024 * 2 + 1024), s>>>(
             static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
     else
-        bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * 2 * 1024 * 4, s>>>(
+        bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * (2 * 1024 * 4 + 1024), s>>>(
             static_cast<const float*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
 }
 
