@@ -409,6 +409,24 @@ aggregate_bitwise_kernel(const uint32_t* __restrict__ planes, const float* __res
                     const uint32_t on = 0u - ((pw1 >> t) & 1u);
                     acc[t] += __uint_as_float((ub & on) ^ (((sgn >> t) & 1u) << 31));
                 }
+            } else if (w <= 8) {
+                // fields of at most 8 bits: each plane word is spread into the 32 field bytes, four bits per
+                // multiply ((nibble * 0x00204081) & 0x01010101 puts bit i of the nibble at bit 0 of byte i)
+                const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
+                uint32_t fb[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) fb[c] = ((((pw1 >> (4 * c)) & 0xFu) * 0x00204081u) & 0x01010101u) << (w - 1);
+                for (int j = 2; j <= w; ++j) {
+                    const uint32_t pw = (word < words) ? pm[(int64_t)j * words + word] : 0u;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) fb[c] |= ((((pw >> (4 * c)) & 0xFu) * 0x00204081u) & 0x01010101u) << (w - j);
+                }
+#pragma unroll
+                for (int t = 0; t < 32; ++t) {
+                    const uint32_t f = (fb[t >> 2] >> (8 * (t & 3))) & 0xFFu;
+                    const float ff = __uint_as_float(0x4B000000u | f) - 8388608.0f;  // exact integer-to-float through 2^23
+                    acc[t] += __uint_as_float(__float_as_uint(ff * unit) ^ (((sgn >> t) & 1u) << 31));
+                }
             } else {
                 const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
                 uint32_t f[32];
