@@ -173,7 +173,9 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_u = pl.take(sizeof(double) * M_max);
     const size_t o_emit = pl.take(sizeof(EmitParams) * M_max);
     const size_t o_tdesc = pl.take(sizeof(uint4) * ws.max_tiles);
-    const size_t o_tcnt = pl.take(sizeof(unsigned) * M_max);
+    const size_t o_tmax = pl.take(sizeof(uint32_t) * ws.max_tiles);
+    const size_t o_wtiles = pl.take(sizeof(uint32_t) * ws.max_tiles);
+    const size_t o_tilen = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_aggoff = pl.take(sizeof(uint32_t) * (agg_tiles + 1) * M_max);
     const size_t o_gmax = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_S = pl.take(sizeof(unsigned long long) * kMaxLevels * ws.stat_ctas * M_max);
@@ -212,7 +214,9 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.u_dev = reinterpret_cast<double*>(base + o_u);
     ws.emit = reinterpret_cast<EmitParams*>(base + o_emit);
     ws.tile_desc = reinterpret_cast<uint4*>(base + o_tdesc);
-    ws.tile_counter = reinterpret_cast<unsigned*>(base + o_tcnt);
+    ws.tile_max = reinterpret_cast<uint32_t*>(base + o_tmax);
+    ws.worker_tiles = reinterpret_cast<uint32_t*>(base + o_wtiles);
+    ws.tile_n = reinterpret_cast<uint32_t*>(base + o_tilen);
     ws.agg_offsets = reinterpret_cast<uint32_t*>(base + o_aggoff);
     ws.gmax_bits = reinterpret_cast<uint32_t*>(base + o_gmax);
     ws.S_partial = reinterpret_cast<unsigned long long*>(base + o_S);
@@ -263,7 +267,7 @@ int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches :
 static const char* const kKernelNames[K_COUNT] = {
     "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "sums_candidates", "cand_pass2", "masked_pass2",
     "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
-    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise"};
+    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
 

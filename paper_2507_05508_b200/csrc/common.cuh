@@ -16,13 +16,10 @@ constexpr uint32_t kKeyNone = 0xFFFFFFFFu;    // threshold above every finite ke
 constexpr uint32_t kNoSlot = 0xFFu;
 
 constexpr int kSweepThreads = 512;            // histogram / masked / norm sweeps
-constexpr int kEmitWorkers = 8;               // warps that count and write; two more warps per block compute the prefixes
-constexpr int kEmitThreads = (kEmitWorkers + 2) * 32;
-constexpr int kEmitBlocksPerSM = 3;
-constexpr int kEmitMaxWorkers = 1024;         // M of one call: the emit kernel keeps every worker's band parameters in shared memory
-constexpr int kEmitRows = 16;                 // 32-bit words per lane per tile (1 fp32 or 2 bf16 elements each)
-constexpr int kEmitStages = 4;                // tiles of one block resident in shared memory
-constexpr int kEmitTile = kEmitWorkers * 32 * kEmitRows;   // words per tile = elements per fp32 tile; bf16: twice as many
+constexpr int kEmitMaxWorkers = 1024;         // M of one call: the emit and averaging kernels keep per-worker offsets in shared memory
+constexpr int kEmitRows = 16;                 // 32-bit words per lane that a warp of the emit kernels holds at a time
+constexpr int kEmitTile = 4096;               // 32-bit words per emit tile (1 fp32 or 2 bf16 elements each); one warp per tile
+constexpr int kEmitTileVecs = kEmitTile / 4;  // 16-byte vectors per tile, for both element types
 constexpr int kAggTile = 4096;                // dense output elements per aggregation tile
 
 // Per-worker selection query: the rank-k element of the total order.
@@ -54,7 +51,7 @@ struct EmitParams {
 enum KernelId {
     K_DRAW_FIXED = 0, K_INIT_QUERIES, K_UNIFORMS, K_HIST1, K_RESOLVE1, K_SUMS_CAND, K_CAND2, K_MASKED2, K_RESOLVE2, K_CAND3,
     K_MASKED3, K_RESOLVE3, K_CAND_SUMS, K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
-    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_COUNT
+    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_TILE_LIST, K_BAND_COUNT, K_BAND_SCAN, K_COUNT
 };
 
 constexpr int kTimingPool = 2048;  // event pairs kept between two reads
@@ -96,9 +93,11 @@ struct Workspace {
     double* delta_all;           // [M][kMaxLevels]
     double* u_dev;               // [M]
     EmitParams* emit;            // [M]
-    uint4* tile_desc;            // [max_tiles] look-back records {C, A, B, state}
+    uint4* tile_desc;            // [M][tiles per worker] per listed tile {C, A, B}: its own counts, then the running totals before it
     int64_t max_tiles;
-    unsigned int* tile_counter;  // ticket counter (entry 0): tiles are numbered in the order they are taken
+    uint32_t* tile_max;          // [M][tiles per worker] largest magnitude key of every emit tile (sweep 1)
+    uint32_t* worker_tiles;      // [M][tiles per worker] the tiles of a worker that can hold band entries, ascending
+    uint32_t* tile_n;            // [M] how many of them
     uint32_t* agg_offsets;       // [M][agg_tiles_max + 1]
     // bit-wise
     uint32_t* gmax_bits;         // [M]
@@ -203,6 +202,13 @@ __device__ __forceinline__ void block_vector_range(int64_t d, int vec, int bx, i
     const int64_t per = (nvec + nb - 1) / nb;
     *v0 = min((int64_t)bx * per, nvec);
     *v1 = min(*v0 + per, nvec);
+}
+
+// Emit tiles of one row: kEmitTile 32-bit words each (one fp32 or two bf16 elements per word).
+inline int emit_tiles_per_worker(int64_t d, int dtype) {
+    const int per_word = (dtype == MLMC_BF16) ? 2 : 1;
+    const int64_t words = (d + per_word - 1) / per_word;
+    return (int)((words + kEmitTile - 1) / kEmitTile);
 }
 
 // Brackets one kernel launch: counts it and, when timing is on, records an event pair on the stream.

@@ -75,29 +75,50 @@ __global__ void uniforms_kernel(double* u_dev, int M, uint64_t seed, uint64_t st
 // -------------------------------------------------------------------------------------------
 // sweep 1: leading-digit histogram of every worker (shared-memory counts, flushed with atomics)
 // -------------------------------------------------------------------------------------------
+// The sweep also records the largest key of every emit tile (kEmitTileVecs consecutive 16-byte vectors of the
+// row): the emit sweep reads only the tiles whose largest key reaches the lower threshold of the drawn band.
+// Block ranges start at a multiple of 32 vectors, so the 32 vectors a warp loads together lie in one tile.
 template <typename T>
 __global__ void __launch_bounds__(kHistThreads, 1)
-hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restrict__ hist1, int* status,
-             int* worker_err) {
+hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restrict__ hist1,
+             uint32_t* __restrict__ tile_max, int tiles_per_worker, int* status, int* worker_err) {
     extern __shared__ uint32_t sh_hist[];
     using Tr = ElemTraits<T>;
     const int m = blockIdx.y;
     for (int b = threadIdx.x; b < kBins1; b += blockDim.x) sh_hist[b] = 0;
     __syncthreads();
     const T* row = g + (int64_t)m * ld;
+    uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker;
     int64_t v0, v1;
-    block_vector_range(d, Tr::kVec, blockIdx.x, gridDim.x, &v0, &v1);
+    {
+        const int64_t nvec = (d + Tr::kVec - 1) / Tr::kVec;
+        const int64_t groups = (nvec + 31) / 32;
+        const int64_t per = (groups + gridDim.x - 1) / gridDim.x;
+        v0 = min((int64_t)blockIdx.x * per * 32, nvec);
+        v1 = min(v0 + per * 32, nvec);
+    }
     bool bad = false;
     auto count_key = [&](uint32_t bits) {
         const uint32_t key = Tr::key(bits);
         bad |= (key >= Tr::kInfKey);
         atomicAdd(&sh_hist[key >> Tr::kShift1], 1u);
     };
+    auto vector_max = [&](const uint4& q) -> uint32_t {  // largest key of one vector
+        if constexpr (Tr::kVec == 4) {
+            return max(max(q.x & 0x7FFFFFFFu, q.y & 0x7FFFFFFFu), max(q.z & 0x7FFFFFFFu, q.w & 0x7FFFFFFFu));
+        } else {
+            const uint32_t a = __vmaxu2(__vmaxu2(q.x & 0x7FFF7FFFu, q.y & 0x7FFF7FFFu),
+                                        __vmaxu2(q.z & 0x7FFF7FFFu, q.w & 0x7FFF7FFFu));
+            return max(a & 0xFFFFu, a >> 16);
+        }
+    };
     // four 16-byte loads per thread are issued before any of them is used: 64 KB in flight per SM
     constexpr int kBatch = 4;
     const int64_t full_end = min(v1, d / Tr::kVec);  // vectors that lie wholly inside the row
+    const int lane = threadIdx.x & 31;
     int64_t v = v0 + threadIdx.x;
-    for (; v + (int64_t)(kBatch - 1) * blockDim.x < full_end; v += (int64_t)kBatch * blockDim.x) {
+    // warp-uniform loop condition (the last lane's last vector is inside): the warp reduces together
+    for (; (v - lane) + 31 + (int64_t)(kBatch - 1) * blockDim.x < full_end; v += (int64_t)kBatch * blockDim.x) {
         uint4 q[kBatch];
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v + (int64_t)j * blockDim.x);
@@ -109,9 +130,18 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
                 count_key(q[j].x & 0xFFFFu); count_key(q[j].x >> 16); count_key(q[j].y & 0xFFFFu); count_key(q[j].y >> 16);
                 count_key(q[j].z & 0xFFFFu); count_key(q[j].z >> 16); count_key(q[j].w & 0xFFFFu); count_key(q[j].w >> 16);
             }
+            const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, vector_max(q[j]));
+            if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitTileVecs], wm);
         }
     }
-    for (; v < v1; v += blockDim.x) for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) { count_key(bits); });
+    for (; v < v1; v += blockDim.x) {
+        uint32_t vm = 0;
+        for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) {
+            count_key(bits);
+            vm = max(vm, Tr::key(bits));
+        });
+        atomicMax(&tmax[v / kEmitTileVecs], vm);
+    }
     if (bad) {
         worker_err[m] = MLMC_ERR_NONFINITE;
         set_status(status, MLMC_ERR_NONFINITE);
@@ -831,17 +861,19 @@ void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStr
 }
 
 void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
+    const int tpw = emit_tiles_per_worker(d, dtype);
     cudaMemsetAsync(ws.hist1, 0, (size_t)M * kBins1 * sizeof(uint32_t), s);
+    cudaMemsetAsync(ws.tile_max, 0, (size_t)M * tpw * sizeof(uint32_t), s);
     const size_t smem = kBins1 * sizeof(uint32_t);
     LaunchScope t(ws, K_HIST1, s);
     if (dtype == MLMC_BF16) {
         const int nb = blocks_per_worker(ws, d, 8, kHistThreads, M, 2);
         hist1_kernel<bf16_t><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const bf16_t*>(g), d, ld, ws.hist1,
-                                                                     ws.status, ws.worker_err);
+                                                                     ws.tile_max, tpw, ws.status, ws.worker_err);
     } else {
         const int nb = blocks_per_worker(ws, d, 4, kHistThreads, M, 2);
         hist1_kernel<float><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.hist1,
-                                                                    ws.status, ws.worker_err);
+                                                                    ws.tile_max, tpw, ws.status, ws.worker_err);
     }
 }
 
