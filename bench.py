@@ -228,11 +228,13 @@ def sweeps_charged(w) -> int:
 
 
 # Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes of its variant, dense bytes).
+# band_count and emit read only the tiles that can hold band entries (a fraction of the row that depends on the
+# drawn levels); they are charged a whole sweep here, so their figure can exceed the copy peak when few tiles are listed.
 def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float):
     mt, mb = msg.get("topk", 0.0), msg.get("bitwise", 0.0)
     table = {
         "hist1": sweep, "sums_candidates": sweep, "masked_pass2": sweep, "masked_pass3": sweep, "norm_sweep": sweep,
-        "emit": sweep + mt, "aggregate_topk": mt + dense,
+        "band_count": sweep, "emit": sweep + mt, "aggregate_topk": mt + dense,
         "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + mb, "aggregate_bitwise": mb + dense,
     }
     return table.get(name)

@@ -48,7 +48,7 @@ typedef enum {
     MLMC_ERR_PROB = -3,      /* some p_l <= 0 or sum p != 1 (Lemma 3.2 needs non-zero probabilities) */
     MLMC_ERR_CAPACITY = -4,  /* device: a Top-k message does not fit out->capacity / planes exceed w_max */
     MLMC_ERR_NONFINITE = -5, /* device: NaN or Inf in g */
-    MLMC_ERR_TIMEOUT = -6,   /* device: a bounded wait between thread blocks gave up */
+    MLMC_ERR_TIMEOUT = -6,   /* reserved (no kernel of this version waits for another thread block) */
     MLMC_ERR_CUDA = -7,      /* a CUDA runtime call failed */
     MLMC_ERR_NOMEM = -8,     /* workspace allocation failed */
     MLMC_ERR_INTERNAL = -9   /* device: a self-check failed (emitted count differs from k_l - k_{l-1}) */
