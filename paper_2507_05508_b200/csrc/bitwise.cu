@@ -307,6 +307,10 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
     };
     const int64_t stride = (int64_t)gridDim.x * warps_per_block;
     int64_t grp = (int64_t)blockIdx.x * warps_per_block + warp;
+    // An entry below gmax 2^-b_l (1 - 2^-20) has fl32(|g| / gmax) < 2^-b_l, so its top b_l code bits and with them
+    // the field of level l are zero.  A row of 32 entries that are all below that bound is not coded at all: in
+    // a gradient with per-layer scales and a few outliers this is most rows of the high levels.
+    const uint32_t zero_below = (gmax > 0.0f) ? __float_as_uint(gmax * ldexpf(1.0f - 0x1.0p-20f, -sc.bits[level])) : 0x7FFFFFFFu;
     fetch(grp, 0);
     for (int it = 0; grp < ngroups; grp += stride, ++it) {
         fetch(grp + stride, (it + 1) & 1);
@@ -314,6 +318,7 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
         __syncwarp();
         const uint8_t* buf = ring + (it & 1) * kGroupBytes;
         uint32_t code[32];  // bit 31 = sign, low bits = field
+        bool coded = false;  // warp-uniform: some row of the group was coded
 #pragma unroll
         for (int s = 0; s < 32; ++s) {
             uint32_t bits;
@@ -321,12 +326,26 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
                 bits = reinterpret_cast<const uint32_t*>(buf)[s * 32 + lane];
             else
                 bits = reinterpret_cast<const uint16_t*>(buf)[s * 32 + lane];
-            const float x = Tr::value(bits);
-            const uint32_t q = (gmax > 0.0f) ? qz.code(__float_as_uint(x) & 0x7FFFFFFFu) : 0u;
-            code[s] = ((q >> shift) & mask) | (__float_as_uint(x) & 0x80000000u);
+            const uint32_t xb = __float_as_uint(Tr::value(bits));
+            code[s] = xb & 0x80000000u;
+            if (__any_sync(0xFFFFFFFFu, (xb & 0x7FFFFFFFu) >= zero_below)) {
+                code[s] |= (qz.code(xb & 0x7FFFFFFFu) >> shift) & mask;
+                coded = true;
+            }
         }
         const int64_t word = grp * 32 + lane;
-        if (w <= 8) {
+        if (!coded) {  // every field of the group is zero: the sign plane by ballots, zero magnitude planes
+            uint32_t sign_w = 0;
+#pragma unroll
+            for (int s = 0; s < 32; ++s) {
+                const uint32_t bs = __ballot_sync(0xFFFFFFFFu, (int)code[s] < 0);
+                if (lane == s) sign_w = bs;
+            }
+            if (word < words) {
+                out[word] = sign_w;
+                for (int j = 1; j <= w; ++j) out[(int64_t)j * words + word] = 0u;
+            }
+        } else if (w <= 8) {
             // Fields of at most 8 bits go through a byte matrix in shared memory: lane L writes the field of each of
             // its 32 rows, then lane r gathers bit b of the 32 bytes of row r, four bytes per multiply
             // (((x >> b) & 0x01010101) * 0x01020408 puts the four bits side by side in bits 24..27).  This costs
@@ -402,30 +421,44 @@ aggregate_bitwise_kernel(const uint32_t* __restrict__ planes, const float* __res
             const int w = sc.width[lv];
             // value of one unit of the field: 2^{-b_l} gmax / p_l
             const float unit = (float)(ldexp((double)gmax[m], -sc.bits[lv]) / p_sel[m]);
+            // A word whose fields are all zero adds +-0 to every entry, which changes nothing: it is skipped.  The
+            // high levels of a heavy-tailed gradient are almost all zero, so whole warps skip.
             if (w == 1) {  // the paper's case: one information bit and one sign bit per entry
-                const uint32_t ub = __float_as_uint(unit);
+                if (pw1 != 0u) {
+                    const uint32_t ub = __float_as_uint(unit);
 #pragma unroll
-                for (int t = 0; t < 32; ++t) {
-                    const uint32_t on = 0u - ((pw1 >> t) & 1u);
-                    acc[t] += __uint_as_float((ub & on) ^ (((sgn >> t) & 1u) << 31));
+                    for (int t = 0; t < 32; ++t) {
+                        const uint32_t on = 0u - ((pw1 >> t) & 1u);
+                        acc[t] += __uint_as_float((ub & on) ^ (((sgn >> t) & 1u) << 31));
+                    }
                 }
             } else if (w <= 8) {
                 // fields of at most 8 bits: each plane word is spread into the 32 field bytes, four bits per
                 // multiply ((nibble * 0x00204081) & 0x01010101 puts bit i of the nibble at bit 0 of byte i)
                 const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
-                uint32_t fb[8];
+                uint32_t pw[8], any = pw1;
+                pw[0] = pw1;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) fb[c] = ((((pw1 >> (4 * c)) & 0xFu) * 0x00204081u) & 0x01010101u) << (w - 1);
-                for (int j = 2; j <= w; ++j) {
-                    const uint32_t pw = (word < words) ? pm[(int64_t)j * words + word] : 0u;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) fb[c] |= ((((pw >> (4 * c)) & 0xFu) * 0x00204081u) & 0x01010101u) << (w - j);
+                for (int j = 2; j <= 8; ++j) {
+                    pw[j - 1] = (j <= w && word < words) ? pm[(int64_t)j * words + word] : 0u;
+                    any |= pw[j - 1];
                 }
+                if (any != 0u) {
+                    uint32_t fb[8] = {};
 #pragma unroll
-                for (int t = 0; t < 32; ++t) {
-                    const uint32_t f = (fb[t >> 2] >> (8 * (t & 3))) & 0xFFu;
-                    const float ff = __uint_as_float(0x4B000000u | f) - 8388608.0f;  // exact integer-to-float through 2^23
-                    acc[t] += __uint_as_float(__float_as_uint(ff * unit) ^ (((sgn >> t) & 1u) << 31));
+                    for (int j = 1; j <= 8; ++j) {
+                        if (j <= w) {
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                fb[c] |= ((((pw[j - 1] >> (4 * c)) & 0xFu) * 0x00204081u) & 0x01010101u) << (w - j);
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < 32; ++t) {
+                        const uint32_t f = (fb[t >> 2] >> (8 * (t & 3))) & 0xFFu;
+                        const float ff = __uint_as_float(0x4B000000u | f) - 8388608.0f;  // exact integer-to-float through 2^23
+                        acc[t] += __uint_as_float(__float_as_uint(ff * unit) ^ (((sgn >> t) & 1u) << 31));
+                    }
                 }
             } else {
                 const uint32_t* pm = planes + (int64_t)m * (1 + w_max) * words;
