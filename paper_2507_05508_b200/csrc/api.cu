@@ -176,6 +176,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_tmax = pl.take(sizeof(uint32_t) * ws.max_tiles);
     const size_t o_wtiles = pl.take(sizeof(uint32_t) * ws.max_tiles);
     const size_t o_tilen = pl.take(sizeof(uint32_t) * M_max);
+    const size_t o_cfloor = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_aggoff = pl.take(sizeof(uint32_t) * (agg_tiles + 1) * M_max);
     const size_t o_gmax = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_S = pl.take(sizeof(unsigned long long) * kMaxLevels * ws.stat_ctas * M_max);
@@ -217,6 +218,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.tile_max = reinterpret_cast<uint32_t*>(base + o_tmax);
     ws.worker_tiles = reinterpret_cast<uint32_t*>(base + o_wtiles);
     ws.tile_n = reinterpret_cast<uint32_t*>(base + o_tilen);
+    ws.cand_floor = reinterpret_cast<uint32_t*>(base + o_cfloor);
     ws.agg_offsets = reinterpret_cast<uint32_t*>(base + o_aggoff);
     ws.gmax_bits = reinterpret_cast<uint32_t*>(base + o_gmax);
     ws.S_partial = reinterpret_cast<unsigned long long*>(base + o_S);

@@ -187,7 +187,8 @@ __device__ void assign_slots(Query* q, int nq, int shift) {
 // For fp32 the kernel also writes the bin table of the second sweep: a bin that holds no threshold maps
 // to its open interval  #{ j : bin_j > b }  (code < 64); a bin that holds one maps to 64 + its slot.
 __global__ void __launch_bounds__(kResolveThreads, 1)
-resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is_bf16, const int* worker_err) {
+resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand_floor, int nq, int is_bf16,
+                const int* worker_err) {
     __shared__ uint32_t sh_warp[32];
     __shared__ int sh_bin[kMaxQueries];
     __shared__ uint32_t sh_slot[kMaxQueries];
@@ -256,6 +257,13 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, int nq, int is
         sh_slot[threadIdx.x] = qq.slot;
     }
     __syncthreads();
+    if (threadIdx.x == 0) {
+        // the smallest key that can be a candidate: the lower edge of the lowest boundary bin (no live query: none)
+        int lowest = kBins1;
+        for (int j = 0; j < nq; ++j)
+            if (sh_bin[j] >= 0 && sh_bin[j] < lowest) lowest = sh_bin[j];
+        cand_floor[m] = (lowest < kBins1) ? ((uint32_t)lowest << 16) : 0xFFFFFFFFu;
+    }
     uint8_t* tab = table1 + (int64_t)m * kBins1;
     for (int i = 0; i < per; ++i) {
         const int b = i * kResolveThreads + threadIdx.x;
@@ -290,7 +298,8 @@ __global__ void __launch_bounds__(kS2Threads, 2)
 sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table, int L,
                        double* __restrict__ sum_partial, uint32_t* __restrict__ region_partial, int sum_ctas,
                        uint32_t* __restrict__ cand_keys, int64_t cand_cap, uint32_t* cand_count, int* cand_overflow,
-                       const int* worker_err, const int* __restrict__ gate) {
+                       const int* worker_err, const int* __restrict__ gate, const uint32_t* __restrict__ tile_max,
+                       int tiles_per_worker, const uint32_t* __restrict__ cand_floor) {
     extern __shared__ __align__(16) uint8_t sh_raw[];
     uint8_t* sh_table = sh_raw;                                                   // [32768]
     uint32_t* sh_stage = reinterpret_cast<uint32_t*>(sh_raw + kBins1);            // [kStage]
@@ -316,9 +325,31 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
     __syncthreads();
     const float* row = g + (int64_t)m * ld;
     uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
-    int64_t v0, v1;
-    block_vector_range(d, 4, blockIdx.x, gridDim.x, &v0, &v1);
-    const int64_t full_end = min(v1, d / 4);  // vectors wholly inside the row
+    // A round is one emit tile (kEmitTileVecs vectors); block b takes rounds b, b + gridDim.x, ...  Without
+    // energies (fixed p) only the candidates matter: a tile whose largest key lies below the lowest boundary bin
+    // holds none and is not read.  Such tiles cluster (whole layers lie below the thresholds), so the rounds are
+    // dealt out round-robin rather than in contiguous ranges.
+    static_assert(kS2Threads * kS2Vecs == kEmitTileVecs, "one round of the sweep is one emit tile");
+    const int64_t v1 = (d + 3) / 4;                                  // vectors of the row
+    const int64_t v0 = min((int64_t)blockIdx.x * kEmitTileVecs, v1);  // this block's first round
+    const int64_t vstep = (int64_t)gridDim.x * kEmitTileVecs;
+    const int64_t full_end = d / 4;  // vectors wholly inside the row
+    // which of the block's rounds hold a candidate, looked up once (rounds past the flag array are swept anyway)
+    constexpr int kWantFlags = 2048;
+    __shared__ uint8_t sh_want[kWantFlags];
+    if (!SUMS) {
+        const uint32_t floor_key = cand_floor[m];
+        const uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker + blockIdx.x;
+        const int64_t nrounds = (v1 - v0 + vstep - 1) / vstep;
+        for (int r = threadIdx.x; r < kWantFlags && r < nrounds; r += kS2Threads)
+            sh_want[r] = tmax[(int64_t)r * gridDim.x] >= floor_key;
+        __syncthreads();
+    }
+    auto wanted = [&](int64_t vb) -> bool {  // block-uniform
+        if (SUMS) return true;
+        const int64_t r = (vb - v0) / vstep;
+        return vb < v1 && (r >= kWantFlags || sh_want[r]);
+    };
 
     auto flush = [&]() {  // called by all threads
         const uint32_t n = sh_n;
@@ -359,9 +390,17 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
     };
 
     uint4 cur[kS2Vecs], nxt[kS2Vecs];
-    load_round(v0, cur);
-    for (int64_t vb = v0; vb < v1; vb += kS2Threads * kS2Vecs) {
-        load_round(vb + kS2Threads * kS2Vecs, nxt);
+    bool want_cur = wanted(v0);
+    if (want_cur) load_round(v0, cur);
+    for (int64_t vb = v0; vb < v1; vb += vstep) {
+        const bool want_nxt = wanted(vb + vstep);
+        if (want_nxt) load_round(vb + vstep, nxt);
+        if (!SUMS && !want_cur) {  // nothing to do in this round: no barrier either (block-uniform)
+            want_cur = want_nxt;
+#pragma unroll
+            for (int j = 0; j < kS2Vecs; ++j) cur[j] = nxt[j];
+            continue;
+        }
 #pragma unroll
         for (int j = 0; j < kS2Vecs; ++j) {
             const int64_t v = vb + j * kS2Threads + threadIdx.x;
@@ -373,6 +412,7 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
         }
         __syncthreads();
         if (sh_n > (uint32_t)kStageSlack) flush();  // uniform: sh_n is read after the barrier; a round adds at most kS2Round
+        want_cur = want_nxt;
 #pragma unroll
         for (int j = 0; j < kS2Vecs; ++j) cur[j] = nxt[j];
     }
@@ -879,8 +919,8 @@ void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int
 
 void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
     LaunchScope t(ws, K_RESOLVE1, s);
-    resolve1_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, ws.table1, L - 1, dtype == MLMC_BF16,
-                                                  ws.worker_err);
+    resolve1_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, ws.table1, ws.cand_floor, L - 1,
+                                                  dtype == MLMC_BF16, ws.worker_err);
 }
 
 static int cand_blocks(const Workspace& ws, int M) {
@@ -898,7 +938,7 @@ void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int6
                             cudaStream_t s) {
     cudaMemsetAsync(ws.cand_count, 0, sizeof(uint32_t) * M, s);
     cudaMemsetAsync(ws.cand_overflow, 0, sizeof(int) * M, s);
-    int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, 2);
+    int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, sums ? 2 : 8);  // without the accumulators four blocks fit an SM
     if (nb > ws.sum_ctas) nb = ws.sum_ctas;
     ws.cur_sum_ctas = nb;
     const size_t smem = s2_smem(L, sums, false);
@@ -906,11 +946,13 @@ void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int6
     if (sums)
         sums_candidates_kernel<true, false><<<dim3(nb, M), kS2Threads, smem, s>>>(
             static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, nullptr, ws.sum_ctas, ws.cand_keys,
-            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr);
+            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr, ws.tile_max,
+            emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor);
     else
         sums_candidates_kernel<false, false><<<dim3(nb, M), kS2Threads, smem, s>>>(
             static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, nullptr, ws.sum_ctas, ws.cand_keys,
-            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr);
+            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr, ws.tile_max,
+            emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor);
 }
 
 // Digit pass 2 or 3: over the candidate keys, and (early exit unless the buffer overflowed) over the full row.
