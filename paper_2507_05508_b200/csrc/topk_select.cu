@@ -77,7 +77,7 @@ __global__ void uniforms_kernel(double* u_dev, int M, uint64_t seed, uint64_t st
 // -------------------------------------------------------------------------------------------
 // The sweep also records the largest key of every emit tile (kEmitTileVecs consecutive 16-byte vectors of the
 // row): the emit sweep reads only the tiles whose largest key reaches the lower threshold of the drawn band.
-// Block ranges start at a multiple of 32 vectors, so the 32 vectors a warp loads together lie in one tile.
+// Chunks start at a multiple of 32 vectors, so the 32 vectors a warp loads together lie in one tile.
 template <typename T>
 __global__ void __launch_bounds__(kHistThreads, 1)
 hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restrict__ hist1,
@@ -89,14 +89,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
     __syncthreads();
     const T* row = g + (int64_t)m * ld;
     uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker;
-    int64_t v0, v1;
-    {
-        const int64_t nvec = (d + Tr::kVec - 1) / Tr::kVec;
-        const int64_t groups = (nvec + 31) / 32;
-        const int64_t per = (groups + gridDim.x - 1) / gridDim.x;
-        v0 = min((int64_t)blockIdx.x * per * 32, nvec);
-        v1 = min(v0 + per * 32, nvec);
-    }
+    const int64_t nvec = (d + Tr::kVec - 1) / Tr::kVec;
     bool bad = false;
     auto count_key = [&](uint32_t bits) {
         const uint32_t key = Tr::key(bits);
@@ -114,11 +107,24 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
     };
     // four 16-byte loads per thread are issued before any of them is used: 64 KB in flight per SM
     constexpr int kBatch = 4;
-    const int64_t full_end = min(v1, d / Tr::kVec);  // vectors that lie wholly inside the row
+    const int64_t full_end = d / Tr::kVec;  // vectors that lie wholly inside the row
     const int lane = threadIdx.x & 31;
-    int64_t v = v0 + threadIdx.x;
-    // warp-uniform loop condition (the last lane's last vector is inside): the warp reduces together
-    for (; (v - lane) + 31 + (int64_t)(kBatch - 1) * blockDim.x < full_end; v += (int64_t)kBatch * blockDim.x) {
+    // Chunks of kBatch * blockDim.x vectors are dealt round-robin to the blocks of a worker (how fast a chunk is
+    // counted depends on how its keys collide in the shared-memory histogram, which differs from layer to layer).
+    const int64_t chunk = (int64_t)kBatch * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * chunk; base < nvec; base += (int64_t)gridDim.x * chunk) {
+        const int64_t v = base + threadIdx.x;
+        if (base + chunk > full_end) {  // the row's last chunk: vector by vector (block-uniform branch)
+            for (int64_t u = v; u < nvec; u += blockDim.x) {
+                uint32_t vm = 0;
+                for_each_in_vector<T>(row, u, d, [&](int64_t, uint32_t bits) {
+                    count_key(bits);
+                    vm = max(vm, Tr::key(bits));
+                });
+                atomicMax(&tmax[u / kEmitTileVecs], vm);
+            }
+            break;
+        }
         uint4 q[kBatch];
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v + (int64_t)j * blockDim.x);
@@ -133,14 +139,6 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
             const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, vector_max(q[j]));
             if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitTileVecs], wm);
         }
-    }
-    for (; v < v1; v += blockDim.x) {
-        uint32_t vm = 0;
-        for_each_in_vector<T>(row, v, d, [&](int64_t, uint32_t bits) {
-            count_key(bits);
-            vm = max(vm, Tr::key(bits));
-        });
-        atomicMax(&tmax[v / kEmitTileVecs], vm);
     }
     if (bad) {
         worker_err[m] = MLMC_ERR_NONFINITE;
