@@ -188,41 +188,52 @@ __global__ void __launch_bounds__(kResolveThreads, 1)
 resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand_floor, int nq, int is_bf16,
                 const int* worker_err) {
     __shared__ uint32_t sh_warp[32];
+    __shared__ uint32_t sh_tot[kResolveThreads], sh_off[kResolveThreads];
     __shared__ int sh_bin[kMaxQueries];
     __shared__ uint32_t sh_slot[kMaxQueries];
     const int m = blockIdx.x;
     uint32_t* S = hist1 + (int64_t)m * kBins1;
     Query* q = queries + m * kMaxQueries;
     constexpr int per = kBins1 / kResolveThreads;  // 32 chunks of 1024 bins; thread t owns bin c * 1024 + t of chunk c
+    static_assert(per == 32 && kResolveThreads == 1024, "the (chunk, warp) totals are scanned by one thread each");
     {
-        // suffix sums S[b] = #{digit >= b}, chunk by chunk from the top, coalesced
+        // suffix sums S[b] = #{digit >= b}, coalesced: 32 chunks of 1024 bins, thread t owns bin c * 1024 + t of
+        // chunk c.  Every warp first scans its 32 bins of every chunk, then one scan over the 32 x 32 (chunk, warp)
+        // totals gives each of them what lies above it: three barriers in all.
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        uint32_t carry = 0;
         uint32_t cnt[per];
 #pragma unroll
         for (int c = 0; c < per; ++c) cnt[c] = S[c * kResolveThreads + threadIdx.x];  // all 32 loads in flight at once
 #pragma unroll
-        for (int c = per - 1; c >= 0; --c) {
-            const int b = c * kResolveThreads + threadIdx.x;
+        for (int c = 0; c < per; ++c) {
             uint32_t v = cnt[c];
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {  // inclusive suffix within the warp
                 const uint32_t y = __shfl_down_sync(0xFFFFFFFFu, v, o);
                 if (lane + o < 32) v += y;
             }
-            if (lane == 0) sh_warp[warp] = v;
-            __syncthreads();
-            uint32_t higher = 0, total = 0;
-#pragma unroll 8
-            for (int w = 0; w < kResolveThreads / 32; ++w) {
-                const uint32_t x = sh_warp[w];
-                total += x;
-                if (w > warp) higher += x;
-            }
-            S[b] = v + higher + carry;
-            carry += total;
-            __syncthreads();
+            cnt[c] = v;
+            if (lane == 0) sh_tot[c * 32 + warp] = v;
         }
+        __syncthreads();
+        // entry e = chunk * 32 + warp, taken by thread e: exclusive suffix sum over the entries in that order
+        const uint32_t x = sh_tot[threadIdx.x];
+        uint32_t v = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_down_sync(0xFFFFFFFFu, v, o);
+            if (lane + o < 32) v += y;
+        }
+        if (lane == 0) sh_warp[warp] = v;  // total of chunk `warp`
+        __syncthreads();
+        uint32_t higher = 0;
+#pragma unroll 8
+        for (int c = 0; c < 32; ++c)
+            if (c > warp) higher += sh_warp[c];
+        sh_off[threadIdx.x] = v - x + higher;
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < per; ++c) S[c * kResolveThreads + threadIdx.x] = cnt[c] + sh_off[c * 32 + warp];
     }
     __syncthreads();
     if (worker_err[m]) return;
@@ -511,14 +522,17 @@ cand_sums_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const
         }
     }
     __syncthreads();
+    // each warp adds up every fourth (interval, side, half) column: four values per lane, then a shuffle tree
     unsigned long long* out = cand_S + (int64_t)m * kMaxLevels * 4;
-    for (int q = 0; q < L * 4; ++q) {
-        unsigned long long* a = sh_S + q * kCandSumThreads;
-        for (int s = kCandSumThreads >> 1; s > 0; s >>= 1) {
-            if (threadIdx.x < s) a[threadIdx.x] += a[threadIdx.x + s];
-            __syncthreads();
-        }
-        if (threadIdx.x == 0 && a[0]) atomicAdd(&out[q], a[0]);  // integer: the order of the blocks does not matter
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int q = warp; q < L * 4; q += kCandSumThreads / 32) {
+        const unsigned long long* a = sh_S + q * kCandSumThreads;
+        unsigned long long x = 0;
+#pragma unroll
+        for (int i = 0; i < kCandSumThreads / 32; ++i) x += a[i * 32 + lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        if (lane == 0 && x) atomicAdd(&out[q], x);  // integer: the order of the blocks does not matter
     }
 }
 
@@ -957,7 +971,7 @@ void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int6
 void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s) {
     const size_t hist_bytes = (size_t)M * kMaxQueries * kBins23 * sizeof(uint32_t);
     const size_t smem = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
-    const int nb_full = blocks_per_worker(ws, d, 4, kSweepThreads, M, 6);
+    const int nb_full = blocks_per_worker(ws, d, 4, kSweepThreads, M, 2);  // fall-back sweeps: a small grid, since they normally exit at once
     const int nb_cand = cand_blocks(ws, M);
     if (pass == 2) {
         cudaMemsetAsync(ws.hist2, 0, hist_bytes, s);
@@ -996,13 +1010,13 @@ void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
 // Band energies of the boundary bins from the candidate keys, and the full-sweep fallback.
 void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
     {
-        const int nb = cand_blocks(ws, M);
+        const int nb = 3 * cand_blocks(ws, M);
         cudaMemsetAsync(ws.cand_S, 0, (size_t)M * kMaxLevels * 4 * sizeof(unsigned long long), s);
         LaunchScope t(ws, K_CAND_SUMS, s);
         cand_sums_kernel<<<dim3(nb, M), kCandSumThreads, (size_t)L * 4 * kCandSumThreads * sizeof(unsigned long long), s>>>(
             ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.queries, L, ws.cand_S, ws.worker_err);
     }
-    int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 4);
+    int nb = blocks_per_worker(ws, d, 4, kSweepThreads, M, 2);
     if (nb > ws.norm_ctas) nb = ws.norm_ctas;
     ws.cur_norm_ctas = nb;
     const size_t smem = (size_t)L * kSweepThreads * sizeof(double);
