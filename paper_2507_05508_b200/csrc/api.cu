@@ -269,7 +269,7 @@ int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches :
 static const char* const kKernelNames[K_COUNT] = {
     "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "sums_candidates", "cand_pass2", "masked_pass2",
     "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
-    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan"};
+    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
 

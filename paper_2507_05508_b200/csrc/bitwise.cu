@@ -262,8 +262,11 @@ __global__ void bit_probs_draw_kernel(BitSchedule sc, const uint32_t* gmax_bits,
 // ---- pack: every warp turns 1024 consecutive entries into 32 words of each plane.
 // The entries of a group are staged in a two-slot shared-memory ring private to the warp: the next group's
 // copy (cp.async) is in flight while the current group is coded and packed.
-template <typename T>
-__global__ void __launch_bounds__(kBitThreads, 2)
+// WIDE = false serves the workers whose drawn level has a field of at most 8 bits, WIDE = true the others (each
+// instance leaves the other's workers alone): the narrow path keeps no per-row state in registers, which the wide
+// path's 32 codes per lane would otherwise force on it.
+template <typename T, bool WIDE>
+__global__ void __launch_bounds__(kBitThreads, WIDE ? 2 : 3)
 bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* __restrict__ gmax_bits,
                 BitSchedule sc, const int32_t* __restrict__ bit_level, uint32_t* __restrict__ planes, int w_max,
                 int64_t words) {
@@ -274,6 +277,7 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
     const int m = blockIdx.y;
     const int level = bit_level[m];
     if (level < 0) return;
+    if ((sc.width[level] > 8) != WIDE) return;  // the other instance's worker
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int warps_per_block = kBitThreads / 32;
     const int64_t ngroups = (words + 31) / 32;  // groups of 32 words = 1024 entries
@@ -317,59 +321,59 @@ bit_pack_kernel(const T* __restrict__ g, int64_t d, int64_t ld, const uint32_t* 
         cp_async_wait<1>();  // this group has landed (the next one may still be in flight)
         __syncwarp();
         const uint8_t* buf = ring + (it & 1) * kGroupBytes;
-        uint32_t code[32];  // bit 31 = sign, low bits = field
-        bool coded = false;  // warp-uniform: some row of the group was coded
-#pragma unroll
-        for (int s = 0; s < 32; ++s) {
+        const int64_t word = grp * 32 + lane;
+        auto entry_bits = [&](int s) -> uint32_t {
             uint32_t bits;
             if constexpr (Tr::kVec == 4)
                 bits = reinterpret_cast<const uint32_t*>(buf)[s * 32 + lane];
             else
                 bits = reinterpret_cast<const uint16_t*>(buf)[s * 32 + lane];
-            const uint32_t xb = __float_as_uint(Tr::value(bits));
-            code[s] = xb & 0x80000000u;
-            if (__any_sync(0xFFFFFFFFu, (xb & 0x7FFFFFFFu) >= zero_below)) {
-                code[s] |= (qz.code(xb & 0x7FFFFFFFu) >> shift) & mask;
-                coded = true;
-            }
-        }
-        const int64_t word = grp * 32 + lane;
-        if (!coded) {  // every field of the group is zero: the sign plane by ballots, zero magnitude planes
-            uint32_t sign_w = 0;
-#pragma unroll
-            for (int s = 0; s < 32; ++s) {
-                const uint32_t bs = __ballot_sync(0xFFFFFFFFu, (int)code[s] < 0);
-                if (lane == s) sign_w = bs;
-            }
-            if (word < words) {
-                out[word] = sign_w;
-                for (int j = 1; j <= w; ++j) out[(int64_t)j * words + word] = 0u;
-            }
-        } else if (w <= 8) {
+            return __float_as_uint(Tr::value(bits));
+        };
+        if constexpr (!WIDE) {
             // Fields of at most 8 bits go through a byte matrix in shared memory: lane L writes the field of each of
             // its 32 rows, then lane r gathers bit b of the 32 bytes of row r, four bytes per multiply
             // (((x >> b) & 0x01010101) * 0x01020408 puts the four bits side by side in bits 24..27).  This costs
             // a quarter of one ballot per row and plane.  The sign plane takes one ballot per row.
             uint32_t sign_w = 0;
+            bool coded = false;  // warp-uniform: some row of the group was coded
 #pragma unroll
             for (int s = 0; s < 32; ++s) {
-                const uint32_t bs = __ballot_sync(0xFFFFFFFFu, (int)code[s] < 0);
+                const uint32_t xb = entry_bits(s);
+                const uint32_t bs = __ballot_sync(0xFFFFFFFFu, (int)xb < 0);
                 if (lane == s) sign_w = bs;
-                bytes[s * 32 + lane] = (uint8_t)code[s];
+                uint32_t f = 0;
+                if (__any_sync(0xFFFFFFFFu, (xb & 0x7FFFFFFFu) >= zero_below)) {
+                    f = (qz.code(xb & 0x7FFFFFFFu) >> shift) & mask;
+                    coded = true;
+                }
+                bytes[s * 32 + lane] = (uint8_t)f;
             }
             __syncwarp();
-            const uint4 lo = reinterpret_cast<const uint4*>(bytes + lane * 32)[0];
-            const uint4 hi = reinterpret_cast<const uint4*>(bytes + lane * 32)[1];
-            const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
             if (word < words) out[word] = sign_w;
-            for (int j = 1; j <= w; ++j) {
-                const int bit = w - j;
-                uint32_t pw = 0;
+            if (coded) {
+                const uint4 lo = reinterpret_cast<const uint4*>(bytes + lane * 32)[0];
+                const uint4 hi = reinterpret_cast<const uint4*>(bytes + lane * 32)[1];
+                const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                for (int j = 1; j <= w; ++j) {
+                    const int bit = w - j;
+                    uint32_t pw = 0;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) pw |= ((((x[c] >> bit) & 0x01010101u) * 0x01020408u) >> 24 & 0xFu) << (4 * c);
-                if (word < words) out[(int64_t)j * words + word] = pw;
+                    for (int c = 0; c < 8; ++c) pw |= ((((x[c] >> bit) & 0x01010101u) * 0x01020408u) >> 24 & 0xFu) << (4 * c);
+                    if (word < words) out[(int64_t)j * words + word] = pw;
+                }
+            } else if (word < words) {  // every field of the group is zero
+                for (int j = 1; j <= w; ++j) out[(int64_t)j * words + word] = 0u;
             }
         } else {
+            uint32_t code[32];  // bit 31 = sign, low bits = field
+#pragma unroll
+            for (int s = 0; s < 32; ++s) {
+                const uint32_t xb = entry_bits(s);
+                code[s] = xb & 0x80000000u;
+                if (__any_sync(0xFFFFFFFFu, (xb & 0x7FFFFFFFu) >= zero_below))
+                    code[s] |= (qz.code(xb & 0x7FFFFFFFu) >> shift) & mask;
+            }
             for (int j = 0; j <= w; ++j) {
                 const int bit = (j == 0) ? 31 : (w - j);
                 uint32_t mine = 0;
@@ -517,8 +521,9 @@ int bit_blocks(const Workspace& ws, int64_t d, int vec, int M, int waves) {
 }  // namespace
 
 int configure_bit_kernels() {
-    if (cudaFuncSetAttribute(bit_pack_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (kBitThreads / 32) * (2 * 1024 * 4 + 1024)) != cudaSuccess)
+    const int smem = (kBitThreads / 32) * (2 * 1024 * 4 + 1024);
+    if (cudaFuncSetAttribute(bit_pack_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(bit_pack_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return MLMC_ERR_CUDA;
     return MLMC_OK;
 }
@@ -587,22 +592,43 @@ void launch_bit_probs_draw(Workspace& ws, int M, const int32_t* b, int L, bool a
         ws.worker_err);
 }
 
+template <typename T>
+static void launch_bit_pack_t(Workspace& ws, const T* g, int64_t d, int M, int64_t ld, const BitSchedule& sc,
+                              const mlmc_bit_msgs& out, cudaStream_t s) {
+    const int64_t words = (d + 31) / 32;
+    const int64_t ngroups = (words + 31) / 32;
+    const int64_t by_work = (ngroups + (kBitThreads / 32) - 1) / (kBitThreads / 32);
+    const size_t smem = (kBitThreads / 32) * (2 * 1024 * sizeof(T) + 1024);
+    int w_top = 0, w_low = 64;
+    for (int l = 0; l < sc.L; ++l) {
+        w_top = sc.width[l] > w_top ? sc.width[l] : w_top;
+        w_low = sc.width[l] < w_low ? sc.width[l] : w_low;
+    }
+    if (w_low <= 8) {  // some level has a field of at most 8 bits
+        int64_t nb = ((int64_t)ws.sm_count * 3 + M - 1) / M;  // persistent: three resident blocks per SM
+        if (nb > by_work) nb = by_work;
+        if (nb < 1) nb = 1;
+        LaunchScope t(ws, K_BIT_PACK, s);
+        bit_pack_kernel<T, false><<<dim3((unsigned)nb, M), kBitThreads, smem, s>>>(g, d, ld, ws.gmax_bits, sc, ws.bit_level,
+                                                                                out.planes, out.w_max, words);
+    }
+    if (w_top > 8) {  // some level has a wider field
+        int64_t nb = ((int64_t)ws.sm_count * 2 + M - 1) / M;  // two resident blocks per SM
+        if (nb > by_work) nb = by_work;
+        if (nb < 1) nb = 1;
+        LaunchScope t(ws, K_BIT_PACK_WIDE, s);
+        bit_pack_kernel<T, true><<<dim3((unsigned)nb, M), kBitThreads, smem, s>>>(g, d, ld, ws.gmax_bits, sc, ws.bit_level,
+                                                                               out.planes, out.w_max, words);
+    }
+}
+
 void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* b, int L,
                      const mlmc_bit_msgs& out, cudaStream_t s) {
     const BitSchedule sc = make_schedule(b, L);
-    const int64_t words = (d + 31) / 32;
-    const int64_t ngroups = (words + 31) / 32;
-    int64_t nb = (ngroups + (kBitThreads / 32) - 1) / (kBitThreads / 32);
-    const int64_t cap = ((int64_t)ws.sm_count * 2 + M - 1) / M;  // persistent: two resident blocks per SM
-    if (nb > cap) nb = cap;
-    if (nb < 1) nb = 1;
-    LaunchScope t(ws, K_BIT_PACK, s);
     if (dtype == MLMC_BF16)
-        bit_pack_kernel<bf16_t><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * (2 * 1024 * 2 + 1024), s>>>(
-            static_cast<const bf16_t*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
+        launch_bit_pack_t<bf16_t>(ws, static_cast<const bf16_t*>(g), d, M, ld, sc, out, s);
     else
-        bit_pack_kernel<float><<<dim3((unsigned)nb, M), kBitThreads, (kBitThreads / 32) * (2 * 1024 * 4 + 1024), s>>>(
-            static_cast<const float*>(g), d, ld, ws.gmax_bits, sc, ws.bit_level, out.planes, out.w_max, words);
+        launch_bit_pack_t<float>(ws, static_cast<const float*>(g), d, M, ld, sc, out, s);
 }
 
 void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const int32_t* b, int L, int M, int64_t d,
