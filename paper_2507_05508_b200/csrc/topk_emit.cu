@@ -24,6 +24,7 @@ namespace {
 constexpr int kBandThreads = 256;               // 8 warps per block, one tile per warp at a time
 constexpr int kBatchWords = kEmitRows * 32;     // words a warp holds in registers at a time
 constexpr int kBatches = kEmitTile / kBatchWords;
+constexpr int kWriteSlots = 3;                  // shared-memory batches per warp of the write pass
 
 // How a 32-bit word of the gradient row maps to elements: one fp32 element, or two bf16 elements
 // (low half first).  A word past the end of the row reads as kPad, whose keys lie above every
@@ -81,6 +82,31 @@ __device__ __forceinline__ void load_batch(const T* __restrict__ row, int64_t d,
                 v = (uint32_t)reinterpret_cast<const uint16_t*>(row)[wi * 2] | 0x7FFF0000u;
             }
             w[i] = v;
+        }
+    }
+}
+
+// Starts the copy of batch `batch` of tile `tile` into a warp's shared-memory slot (kBatchWords words, word i at
+// slot[i]): 16-byte asynchronous copies, or plain padded stores for the ragged end of the row.
+template <typename T>
+__device__ __forceinline__ void copy_batch_async(const T* __restrict__ row, int64_t d, int64_t tile, int batch, int lane,
+                                                 uint32_t* slot) {
+    using EW = EmitWord<T>;
+    const int64_t w0 = tile * kEmitTile + (int64_t)batch * kBatchWords;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(row) + w0;
+    if ((w0 + kBatchWords) * EW::S <= d) {
+#pragma unroll
+        for (int c = lane; c < kBatchWords / 4; c += 32) cp_async_16(slot + c * 4, words + c * 4);
+    } else {
+        for (int i = lane; i < kBatchWords; i += 32) {
+            const int64_t wi = w0 + i;
+            uint32_t v = EW::kPad;
+            if ((wi + 1) * EW::S <= d) {
+                v = __ldg(words + i);
+            } else if (EW::S == 2 && wi * 2 < d) {  // odd bf16 tail: only the low half exists
+                v = (uint32_t)reinterpret_cast<const uint16_t*>(row)[wi * 2] | 0x7FFF0000u;
+            }
+            slot[i] = v;
         }
     }
 }
@@ -311,14 +337,14 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
                   uint32_t* __restrict__ idx_out, float* __restrict__ val_out, int64_t capacity) {
     using EW = EmitWord<T>;
     constexpr int S = EW::S;
-    extern __shared__ uint32_t sh_off[];  // [M + 1]
-    // a batch that holds band entries is parked here so that its rows can be addressed by a run-time index;
-    // every lane reads back only the words it stored itself
-    __shared__ uint32_t sh_stage[kBandThreads / 32][kBatchWords];
+    // every warp stages its batches in a ring of three shared-memory slots: two copies are in flight while a
+    // batch is ranked, and the rows of a batch can be addressed by a run-time index
+    extern __shared__ __align__(16) uint32_t sh_dyn[];  // [warps][3][kBatchWords] ring, then sh_off[M + 1]
+    uint32_t* sh_off = sh_dyn + (kBandThreads / 32) * kWriteSlots * kBatchWords;
     list_offsets(tile_n, M, sh_off);
     const uint32_t total = sh_off[M];
     const int lane = threadIdx.x & 31;
-    uint32_t* stage = sh_stage[threadIdx.x >> 5] + lane;
+    uint32_t* ring = sh_dyn + (threadIdx.x >> 5) * kWriteSlots * kBatchWords;
     const uint32_t lt = (1u << lane) - 1u;
     const uint32_t warps = gridDim.x * (kBandThreads / 32);
     for (uint32_t f = blockIdx.x * (kBandThreads / 32) + (threadIdx.x >> 5); f < total; f += warps) {
@@ -334,11 +360,22 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
         float* val_w = val_out + (int64_t)m * capacity;
         const uint4 pre = __ldg(&rec[(int64_t)m * tiles_per_worker + j]);
         uint32_t rC = pre.x, rA = pre.y, rB = pre.z;  // running totals before the current batch
-        uint32_t cur[kEmitRows], nxt[kEmitRows];
-        load_batch<T>(row, d, tile, 0, lane, cur);
+        __syncwarp();  // the previous tile's last batches have been read by every lane
+        copy_batch_async<T>(row, d, tile, 0, lane, ring);
+        cp_async_commit();
+        copy_batch_async<T>(row, d, tile, 1, lane, ring + kBatchWords);
+        cp_async_commit();
 #pragma unroll 1
         for (int b = 0; b < kBatches; ++b) {
-            if (b + 1 < kBatches) load_batch<T>(row, d, tile, b + 1, lane, nxt);
+            __syncwarp();  // batch b - 1 has been read by every lane: its slot takes batch b + 2
+            if (b + 2 < kBatches) copy_batch_async<T>(row, d, tile, b + 2, lane, ring + ((b + 2) % kWriteSlots) * kBatchWords);
+            cp_async_commit();  // one group per step, empty at the end of the tile
+            cp_async_wait<2>();  // batch b has landed
+            __syncwarp();
+            const uint32_t* slot = ring + (b % kWriteSlots) * kBatchWords + lane;
+            uint32_t cur[kEmitRows];
+#pragma unroll
+            for (int r = 0; r < kEmitRows; ++r) cur[r] = slot[r * 32];
             uint32_t a1, b1;
             const uint32_t flags = batch_flags<T>(cur, Tb, Ta, &a1, &b1);
             const uint32_t rowany = __reduce_or_sync(0xFFFFFFFFu, flags);
@@ -358,15 +395,13 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
                 uint32_t tA = rA, tB = rB;  // tie ranks, advanced row by row on the ties path
                 const uint32_t e0 = (uint32_t)((tile * kEmitTile + (int64_t)b * kBatchWords + lane) * S);
                 uint32_t rows = (rowany | (rowany >> 16)) & 0xFFFFu;  // rows that hold a closed-range key
-#pragma unroll
-                for (int r = 0; r < kEmitRows; ++r) stage[r * 32] = cur[r];
                 // a rolled loop over the rows that matter: the body is long, unrolling it 16 times would not fit the
                 // instruction cache
 #pragma unroll 1
                 while (rows) {
                     const int i = __ffs(rows) - 1;
                     rows &= rows - 1u;
-                    const uint32_t w = stage[i * 32];
+                    const uint32_t w = slot[i * 32];
                     bool em[S];
                     uint32_t me[S];
                     if (!ties) {
@@ -422,10 +457,9 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
                 }
                 rC += myC; rA += myA; rB += myB;
             }
-#pragma unroll
-            for (int i = 0; i < kEmitRows; ++i) cur[i] = nxt[i];
         }
     }
+    cp_async_wait<0>();
 }
 
 // offsets[m][t] = first message entry of worker m whose index is >= t * kAggTile  (t = 0..ntiles)
@@ -488,7 +522,14 @@ aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict_
 
 }  // namespace
 
-int configure_emit_kernels() { return MLMC_OK; }  // no kernel of this file needs more than the default shared memory
+int configure_emit_kernels() {  // the write pass: 48 KB ring + the list offsets of up to kEmitMaxWorkers workers
+    const int smem = (kBandThreads / 32) * kWriteSlots * kBatchWords * (int)sizeof(uint32_t) +
+                     (kEmitMaxWorkers + 1) * (int)sizeof(uint32_t);
+    if (cudaFuncSetAttribute(band_write_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(band_write_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    return MLMC_OK;
+}
 
 void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const mlmc_topk_msgs& out,
                  cudaStream_t s) {
@@ -517,12 +558,13 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
         band_scan_kernel<<<M, kListThreads, 0, s>>>(ws.tile_desc, tpw, ws.tile_n, ws.emit, ws.status);
     }
     LaunchScope t(ws, K_EMIT, s);
+    const size_t smem_w = smem + (size_t)(kBandThreads / 32) * kWriteSlots * kBatchWords * sizeof(uint32_t);
     if (dtype == MLMC_BF16)
-        band_write_kernel<bf16_t><<<(unsigned)grid, kBandThreads, smem, s>>>(
+        band_write_kernel<bf16_t><<<(unsigned)grid, kBandThreads, smem_w, s>>>(
             static_cast<const bf16_t*>(g), d, ld, tpw, ws.worker_tiles, ws.tile_n, M, ws.emit, ws.tile_desc, out.idx,
             out.val, out.capacity);
     else
-        band_write_kernel<float><<<(unsigned)grid, kBandThreads, smem, s>>>(
+        band_write_kernel<float><<<(unsigned)grid, kBandThreads, smem_w, s>>>(
             static_cast<const float*>(g), d, ld, tpw, ws.worker_tiles, ws.tile_n, M, ws.emit, ws.tile_desc, out.idx,
             out.val, out.capacity);
 }
