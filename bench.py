@@ -219,12 +219,18 @@ class Runner:
         self.B.mlmc_destroy(self.ctx)
 
 
-def sweeps_charged(w) -> int:
-    """Gradient sweeps the method needs (a true data dependence separates them): select -> emit for Top-k,
-    max -> pack for fixed-p bit-wise, max -> field energies -> pack for adaptive bit-wise."""
+def sweeps_charged(w, emit_read_frac=None) -> float:
+    """Gradient sweeps charged to the step: what the method needs (a true data dependence separates them: select ->
+    emit for Top-k, max -> pack for fixed-p bit-wise, max -> field energies -> pack for adaptive bit-wise), or what
+    the kernels moved where that is less.  Top-k moves one whole histogram sweep, for adaptive fp32 a second whole
+    sweep, and two passes over the listed tiles (emit_read_frac of the row each); the fixed-p candidate sweep,
+    which also skips tiles, is counted as nothing, so the figure is a lower bound of the bytes moved."""
     if w.kind == "topk":
-        return 2
-    return 3 if w.adaptive else 2
+        if emit_read_frac is None:
+            return 2.0
+        moved = 1.0 + (1.0 if (w.adaptive and w.dtype != "bf16") else 0.0) + 2.0 * emit_read_frac
+        return min(2.0, moved)
+    return 3.0 if w.adaptive else 2.0
 
 
 # Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes of its variant, dense bytes).
@@ -289,10 +295,16 @@ def run_cuda(args):
 
     # message volume: average over a few steps outside the timed region (levels are redrawn every step)
     probe = min(args.steps, 8)
+    listed_acc, listed_n = 0.0, 0
     for i in range(probe):
         r.step(args.warmup + i)
         for kind, v in r.message_bytes().items():
             msg_acc[kind] = msg_acc.get(kind, 0.0) + v
+        if any(x.kind == "topk" for x in subs):
+            listed, tiles = B.mlmc_read_listed_tiles(r.ctx, w.M)
+            listed_acc += sum(listed) / float(max(1, tiles * w.M))
+            listed_n += 1
+    emit_read_frac = (listed_acc / listed_n) if listed_n else None
     msg_by_kind = {kind: v / probe for kind, v in msg_acc.items()}
     msg_bytes = sum(msg_by_kind.values())
 
@@ -307,7 +319,7 @@ def run_cuda(args):
                 "frac": round(achieved / peak, 4), "peak_source": peak_kind,
                 "traffic": None if ratio is None else ratio * dom_bytes,
                 "alg_bytes_per_launch": dom_bytes, "avg_launch_ms": round(dom_avg_s * 1e3, 4)}
-    b_alg = sum(sweeps_charged(x) * sweep_bytes + dense_bytes for x in subs) + 2 * msg_bytes
+    b_alg = sum(sweeps_charged(x, emit_read_frac) * sweep_bytes + dense_bytes for x in subs) + 2 * msg_bytes
     step_frac = b_alg / (ms_per_step * 1e-3) / 1e9 / peak
     kernels = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] / args.steps,
                    "share": round(v[0] / sum(x[0] for x in per_kernel.values()), 4)}
@@ -355,7 +367,8 @@ def run_cuda(args):
             "config": {"workload": describe(subs) + f", L={r.L}", "l2_policy": "inputs larger than L2: "
                        f"{sweep_bytes / 1e6:.0f} MB per sweep, 2 batches alternated", "parallelism": "replicas only"},
             "elements_per_s": round(world * len(subs) * w.M * w.d / (ms_per_step * 1e-3), 1),
-            "step_roofline": {"alg_bytes_per_step": b_alg, "sweeps_charged": [sweeps_charged(x) for x in subs],
+            "step_roofline": {"alg_bytes_per_step": b_alg, "sweeps_charged": [round(sweeps_charged(x, emit_read_frac), 3) for x in subs],
+                              "emit_tiles_read_frac": None if emit_read_frac is None else round(emit_read_frac, 4),
                               "message_bytes_per_step": msg_bytes, "frac_of_peak": round(step_frac, 4),
                               "frac_of_8TBs": round(b_alg / (ms_per_step * 1e-3) / 8e12, 4)},
             "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "e2e": e2e,

@@ -14,7 +14,8 @@
  *  - Pointers are DEVICE pointers unless marked "host".  The caller owns every buffer; the library
  *    only owns the scratch workspace inside mlmc_ctx.
  *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default
- *    stream).  Nothing synchronises except mlmc_create, mlmc_destroy, mlmc_get_status and mlmc_read_u.
+ *    stream).  Nothing synchronises except mlmc_create, mlmc_destroy, mlmc_get_status, mlmc_read_u and
+ *    mlmc_read_listed_tiles.
  *  - The int return value reports host-side checks made before any launch (arguments, schedule,
  *    probabilities).  Conditions found on the device (message capacity, non-finite input, a bounded
  *    wait that gave up) are written to a sticky status word read by mlmc_get_status; the affected
@@ -104,6 +105,14 @@ int mlmc_timing_read(mlmc_ctx* ctx, double* total_ms, int64_t* launches, void* s
 /* The uniforms of the level draw for workers 0..M-1 at (seed, step), computed on the device and
  * copied to u_host[M].  Synchronous; for checking the counter generator against known answers. */
 int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream);
+
+/* How much of every row the last mlmc_compress_topk on this context read when it emitted the bands (the
+ * band of ranks (k_{l-1}, k_l] of Sec. 3.2): the emission reads only the tiles of 4096 32-bit words (4096 fp32
+ * or 8192 bf16 entries) whose largest magnitude reaches the band's lower threshold, twice each.
+ *   listed_host  host uint32 [M]: tiles of worker m that were read.
+ *   tiles_host   host int64: tiles in one row.
+ * Synchronous (copies from the device and waits for the stream); a measurement aid, not part of the method. */
+int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t* tiles_host, void* stream);
 
 /* Level probabilities and residual norms (Lemma 3.4; Alg. 3 "Compute p^l = Delta^l / sum Delta").
  *   kind   MLMC_TOPK: sched = host int64 k[L];  MLMC_BITWISE: sched = host int64 b[L].

@@ -22,7 +22,7 @@ MLMC_ERR_ARG, MLMC_ERR_SCHEDULE, MLMC_ERR_PROB, MLMC_ERR_CAPACITY = -1, -2, -3, 
 MLMC_ERR_NONFINITE, MLMC_ERR_TIMEOUT, MLMC_ERR_CUDA, MLMC_ERR_NOMEM, MLMC_ERR_INTERNAL = -5, -6, -7, -8, -9
 MLMC_MAX_LEVELS = 32
 
-EXPORTS = ["mlmc_create", "mlmc_destroy", "mlmc_get_status", "mlmc_launch_count", "mlmc_read_u",
+EXPORTS = ["mlmc_create", "mlmc_destroy", "mlmc_get_status", "mlmc_launch_count", "mlmc_read_u", "mlmc_read_listed_tiles",
            "mlmc_kernel_count", "mlmc_kernel_name", "mlmc_timing_enable", "mlmc_timing_read",
            "mlmc_level_probs", "mlmc_compress_topk", "mlmc_compress_bitwise", "mlmc_aggregate",
            "mlmc_aggregate_topk_noalloc"]
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
         L.mlmc_launch_count.argtypes = [vp]
         L.mlmc_launch_count.restype = i64
         L.mlmc_read_u.argtypes = [vp, u64, u64, i32, vp, vp]
+        L.mlmc_read_listed_tiles.argtypes = [vp, i32, vp, vp, vp]
         L.mlmc_level_probs.argtypes = [vp, vp, i32, i64, i32, i64, i32, vp, i32, vp, vp, vp, vp]
         L.mlmc_compress_topk.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_compress_bitwise.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
@@ -144,6 +145,14 @@ def mlmc_read_u(ctx, seed: int, step: int, M: int):
     buf = (C.c_double * M)()
     _check(lib().mlmc_read_u(ctx, seed, step, M, buf, _stream()), "mlmc_read_u")
     return list(buf)
+
+
+def mlmc_read_listed_tiles(ctx, M: int):
+    """(tiles read per worker by the last Top-k emission, tiles per row)."""
+    buf = (C.c_uint32 * M)()
+    tiles = C.c_int64(0)
+    _check(lib().mlmc_read_listed_tiles(ctx, M, buf, C.byref(tiles), _stream()), "mlmc_read_listed_tiles")
+    return list(buf), int(tiles.value)
 
 
 def _g_args(g: torch.Tensor):

@@ -136,6 +136,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.sm_count = prop.multiProcessorCount;
     ws.launches = 0;
     ws.timing = false;
+    ws.last_emit_tiles = 0;
     ws.timing_used = 0;
     ws.ev_start = ws.ev_stop = nullptr;
     ws.ev_id = nullptr;
@@ -318,6 +319,16 @@ int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_ho
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     launch_uniforms(ctx->ws, M, seed, step, s);
     if (cudaMemcpyAsync(u_host, ctx->ws.u_dev, sizeof(double) * M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    return finish(cudaStreamSynchronize(s));
+}
+
+int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t* tiles_host, void* stream) {
+    if (!ctx || !listed_host || !tiles_host || M < 1 || M > ctx->ws.M_max) return MLMC_ERR_ARG;
+    DeviceGuard guard(ctx->ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    *tiles_host = ctx->ws.last_emit_tiles;
+    if (cudaMemcpyAsync(listed_host, ctx->ws.tile_n, sizeof(uint32_t) * M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return MLMC_ERR_CUDA;
     return finish(cudaStreamSynchronize(s));
 }

@@ -98,6 +98,7 @@ struct Workspace {
     uint32_t* tile_max;          // [M][tiles per worker] largest magnitude key of every emit tile (sweep 1)
     uint32_t* worker_tiles;      // [M][tiles per worker] the tiles of a worker that can hold band entries, ascending
     uint32_t* tile_n;            // [M] how many of them
+    int64_t last_emit_tiles;     // tiles per row of the last emission (host side, for mlmc_read_listed_tiles)
     uint32_t* cand_floor;        // [M] smallest key that can be a candidate of sweep 2 (lower edge of the lowest boundary bin)
     uint32_t* agg_offsets;       // [M][agg_tiles_max + 1]
     // bit-wise

@@ -535,6 +535,7 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
                  cudaStream_t s) {
     const int tpw = emit_tiles_per_worker(d, dtype);
     const int64_t most = (int64_t)tpw * M;  // listed tiles at most
+    ws.last_emit_tiles = tpw;
     {
         LaunchScope t(ws, K_TILE_LIST, s);
         tile_list_kernel<<<M, kListThreads, 0, s>>>(ws.tile_max, tpw, ws.emit, dtype == MLMC_BF16 ? 0x7F80u : 0x7F800000u,
