@@ -91,11 +91,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
     uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker;
     const int64_t nvec = (d + Tr::kVec - 1) / Tr::kVec;
     bool bad = false;
-    auto count_key = [&](uint32_t bits) {
-        const uint32_t key = Tr::key(bits);
-        bad |= (key >= Tr::kInfKey);
-        atomicAdd(&sh_hist[key >> Tr::kShift1], 1u);
-    };
+    auto count_key = [&](uint32_t bits) { atomicAdd(&sh_hist[Tr::key(bits) >> Tr::kShift1], 1u); };  // Inf / NaN: see the maxima
     auto vector_max = [&](const uint4& q) -> uint32_t {  // largest key of one vector
         if constexpr (Tr::kVec == 4) {
             return max(max(q.x & 0x7FFFFFFFu, q.y & 0x7FFFFFFFu), max(q.z & 0x7FFFFFFFu, q.w & 0x7FFFFFFFu));
@@ -121,6 +117,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
                     count_key(bits);
                     vm = max(vm, Tr::key(bits));
                 });
+                bad |= vm >= Tr::kInfKey;
                 atomicMax(&tmax[u / kEmitTileVecs], vm);
             }
             break;
@@ -137,6 +134,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
                 count_key(q[j].z & 0xFFFFu); count_key(q[j].z >> 16); count_key(q[j].w & 0xFFFFu); count_key(q[j].w >> 16);
             }
             const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, vector_max(q[j]));
+            bad |= wm >= Tr::kInfKey;  // a non-finite entry shows in the largest key of its warp
             if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitTileVecs], wm);
         }
     }
