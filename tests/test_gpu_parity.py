@@ -240,6 +240,38 @@ def test_topk_single_level_is_identity(B, ora, ctx):
     check_topk(B, ora, ctx, g, [4097], None, 0, 0)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_emission_reads_only_tiles_that_can_hold_band_entries(B, ctx, dtype):
+    """The emission lists, per worker, the tiles (4096 32-bit words) whose largest magnitude reaches the band's lower
+    threshold.  The list must cover every tile that holds a band entry, stay within the row, and be the whole row
+    for the last level (whose lower threshold is zero); a gradient with one loud layer lists few tiles."""
+    per_word = 2 if dtype == "bf16" else 1
+    tile = 4096 * per_word
+    M, d = 4, 40 * tile + 123
+    rng = np.random.default_rng(5)
+    g_np = (rng.standard_normal((M, d)) * 1e-3).astype(np.float32)
+    g_np[:, 7 * tile:9 * tile] *= 1e3                       # one loud layer: tiles 7 and 8
+    g = to_dev(g_np)
+    if dtype == "bf16":
+        g = padded(g.to(torch.bfloat16), 8)
+    k = [64, 1024, d]
+    out = B.TopkBuffers(M, d)
+    tiles_in_row = (d + tile - 1) // tile
+    for step, p in ((0, [0.98, 0.01, 0.01]), (1, [0.01, 0.98, 0.01]), (2, [0.005, 0.005, 0.99])):
+        B.mlmc_compress_topk(ctx, g, k, p, 11, step, out)
+        assert B.mlmc_get_status(ctx) == B.MLMC_OK
+        listed, tiles = B.mlmc_read_listed_tiles(ctx, M)
+        assert tiles == tiles_in_row
+        for m in range(M):
+            n, lv = int(out.count[m]), int(out.level[m])
+            touched = torch.unique((out.idx[m, :n].to(torch.int64) & 0xFFFFFFFF) // tile).numel()
+            assert touched <= listed[m] <= tiles
+            if lv == 2:
+                assert listed[m] == tiles                   # everything below k_1: every tile can hold entries
+            else:
+                assert listed[m] <= 4                       # the loud layer (two tiles, at most one more on each side)
+
+
 def test_level_probs(B, ora, ctx):
     w = wl.shrink(wl.C5A, 600_000, 4)
     k = wl.topk_schedule(w)
