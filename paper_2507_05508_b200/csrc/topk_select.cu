@@ -697,10 +697,12 @@ norm_sweep_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const Quer
 }
 
 // bf16: every key is a histogram bin, so the open-interval sums follow from the counts exactly.
+// Per interval every warp adds up its 32 threads' shares by shuffles; after one barrier thread l adds the 32 warp
+// sums of interval l in warp order (a fixed order: reproducible).
 __global__ void __launch_bounds__(kResolveThreads, 1)
 norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query* queries, int L,
                            double* band_partial, int norm_ctas, const int* worker_err) {
-    __shared__ double sh_red[kResolveThreads];
+    __shared__ double sh_part[kMaxLevels][kResolveThreads / 32];
     __shared__ uint32_t sh_thr[kMaxQueries];
     const int m = blockIdx.x;
     if (worker_err[m]) return;
@@ -709,29 +711,36 @@ norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query*
         sh_thr[threadIdx.x] = (threadIdx.x < L - 1) ? queries[m * kMaxQueries + threadIdx.x].T : 0u;
     __syncthreads();
     constexpr int per = kBins1 / kResolveThreads;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // this thread's keys (coalesced over the block) with their counts and squares, once
+    uint32_t cnt[per];
+#pragma unroll
+    for (int i = 0; i < per; ++i) {
+        const uint32_t key = i * kResolveThreads + threadIdx.x;
+        cnt[i] = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
+    }
     for (int l = 0; l < L; ++l) {
         // open interval l: T_l < key < T_{l-1}   (T_{-1} = +inf, T_{L-1} = -1: everything below)
         const uint32_t hi = (l == 0) ? 0xFFFFFFFFu : sh_thr[l - 1];
         const int64_t lo = (l == L - 1) ? -1 : (int64_t)sh_thr[l];
         double acc = 0.0;
+#pragma unroll
         for (int i = 0; i < per; ++i) {
-            const uint32_t key = i * kResolveThreads + threadIdx.x;  // coalesced over the block
-            if ((int64_t)key > lo && key < hi) {
-                const uint32_t cnt = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
-                if (cnt) {  // empty bins include the Inf/NaN encodings, whose value must not enter the sum
-                    const double x = (double)__uint_as_float(key << 16);
-                    acc = fma((double)cnt, x * x, acc);
-                }
+            const uint32_t key = i * kResolveThreads + threadIdx.x;
+            if ((int64_t)key > lo && key < hi && cnt[i]) {  // empty bins include the Inf/NaN encodings, whose value must not enter the sum
+                const double x = (double)__uint_as_float(key << 16);
+                acc = fma((double)cnt[i], x * x, acc);
             }
         }
-        sh_red[threadIdx.x] = acc;
-        __syncthreads();
-        for (int s = kResolveThreads >> 1; s > 0; s >>= 1) {
-            if (threadIdx.x < s) sh_red[threadIdx.x] += sh_red[threadIdx.x + s];
-            __syncthreads();
-        }
-        if (threadIdx.x == 0) band_partial[((int64_t)m * norm_ctas) * kMaxLevels + l] = sh_red[0];
-        __syncthreads();
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) sh_part[l][warp] = acc;
+    }
+    __syncthreads();
+    if (threadIdx.x < L) {
+        double tot = 0.0;
+        for (int w = 0; w < kResolveThreads / 32; ++w) tot += sh_part[threadIdx.x][w];
+        band_partial[((int64_t)m * norm_ctas) * kMaxLevels + threadIdx.x] = tot;
     }
 }
 
