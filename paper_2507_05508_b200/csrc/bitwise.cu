@@ -29,16 +29,12 @@ struct BitSchedule {
 // 24-bit significands is never closer than 2^-49 (relative) to the midpoint of two fp32 numbers, the fp64
 // product is within 2^-52 of it, so this rounding is the same as that of the fp32 division.
 struct Quantiser {
-    double inv;     // fl64(1 / gmax)
-    float gmax;
-    float two_b;    // 2^B
-    uint32_t qmax;  // 2^B - 1
+    double inv_scaled;  // fl64(1 / gmax) * 2^B
+    uint32_t qmax;      // 2^B - 1
     bool widen_by_bits;  // gmax >= 2^-100: an fp32 operand below the normal range cannot reach q = 1, so its
                          // fp64 image may be built from the bit pattern as if it were normal
     __device__ __forceinline__ Quantiser(float g, int B) {
-        inv = g > 0.0f ? 1.0 / (double)g : 0.0;
-        gmax = g;
-        two_b = (float)(1u << B);
+        inv_scaled = g > 0.0f ? ldexp(1.0 / (double)g, B) : 0.0;
         qmax = (1u << B) - 1u;
         widen_by_bits = g >= 0x1.0p-100f;
     }
@@ -48,9 +44,10 @@ struct Quantiser {
             x = __hiloint2double((int)((mag_bits >> 3) + 0x38000000u), (int)(mag_bits << 29));
         else
             x = (double)__uint_as_float(mag_bits);
-        const float e = (float)(x * inv);              // = fl32(|g| / gmax)
-        const float scaled = __fmul_rn(e, two_b);      // exact power-of-two scaling
-        return min(__float2uint_rz(scaled), qmax);     // truncation: the lower bits are discarded
+        // fl32(|g| / gmax) * 2^B in one rounding: scaling by a power of two commutes with both roundings (a
+        // quotient so small that its fp32 image would be subnormal has the code 0 either way)
+        const float scaled = (float)(x * inv_scaled);
+        return min(__float2uint_rz(scaled), qmax);  // truncation: the lower bits are discarded
     }
 };
 
