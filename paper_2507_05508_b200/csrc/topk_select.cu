@@ -296,37 +296,29 @@ constexpr int kStage = kS2Round + kStageSlack;                // staged candidat
 
 // table: bin -> code.  code < 64: the bin lies wholly inside open interval `code` (between two thresholds);
 // code >= 64: the bin may hold a threshold, its keys are compacted into the candidate buffer.
-// SUMS: per-interval energy of the threshold-free bins (adaptive p).  COUNTS: per-interval element counts
-// (needed when the table comes from a sample and has to be verified).  gate (optional): only workers with
-// gate[m] != 0 are processed.  Loads are double-buffered in registers: the next round's four 16-byte
-// vectors are in flight while the current round is processed.
-template <bool SUMS, bool COUNTS>
+// SUMS: per-interval energy of the threshold-free bins (adaptive p).  Loads are double-buffered in registers:
+// the next round's 16-byte vectors are in flight while the current round is processed.
+template <bool SUMS>
 __global__ void __launch_bounds__(kS2Threads, 2)
 sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table, int L,
-                       double* __restrict__ sum_partial, uint32_t* __restrict__ region_partial, int sum_ctas,
+                       double* __restrict__ sum_partial, int sum_ctas,
                        uint32_t* __restrict__ cand_keys, int64_t cand_cap, uint32_t* cand_count, int* cand_overflow,
-                       const int* worker_err, const int* __restrict__ gate, const uint32_t* __restrict__ tile_max,
+                       const int* worker_err, const uint32_t* __restrict__ tile_max,
                        int tiles_per_worker, const uint32_t* __restrict__ cand_floor) {
     extern __shared__ __align__(16) uint8_t sh_raw[];
     uint8_t* sh_table = sh_raw;                                                   // [32768]
     uint32_t* sh_stage = reinterpret_cast<uint32_t*>(sh_raw + kBins1);            // [kStage]
     double* sh_acc = reinterpret_cast<double*>(sh_raw + kBins1 + kStage * 4);     // [L][kS2Threads]  (SUMS)
-    uint32_t* sh_cnt = reinterpret_cast<uint32_t*>(sh_raw + kBins1 + kStage * 4 +
-                                                   (SUMS ? (size_t)L * kS2Threads * sizeof(double) : 0));  // [L][kS2Threads]
     __shared__ uint32_t sh_n;
     __shared__ uint32_t sh_base;
-    __shared__ uint32_t sh_tot[kMaxLevels];
     const int m = blockIdx.y;
-    if (worker_err[m] || (gate && !gate[m])) return;
+    if (worker_err[m]) return;
     {
         const uint4* src = reinterpret_cast<const uint4*>(table + (int64_t)m * kBins1);
         uint4* dst = reinterpret_cast<uint4*>(sh_table);
         for (int i = threadIdx.x; i < kBins1 / 16; i += kS2Threads) dst[i] = src[i];
         if (SUMS)
             for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_acc[i] = 0.0;
-        if (COUNTS)
-            for (int i = threadIdx.x; i < L * kS2Threads; i += kS2Threads) sh_cnt[i] = 0u;
-        if (threadIdx.x < kMaxLevels) sh_tot[threadIdx.x] = 0u;
         if (threadIdx.x == 0) sh_n = 0;
     }
     __syncthreads();
@@ -383,7 +375,6 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
                 double* a = &sh_acc[code * kS2Threads + threadIdx.x];
                 *a = fma(x, x, *a);
             }
-            if (COUNTS) sh_cnt[code * kS2Threads + threadIdx.x] += 1u;
         } else {
             sh_stage[atomicAdd(&sh_n, 1u)] = key;
         }
@@ -433,14 +424,6 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
             }
             if (threadIdx.x == 0) sum_partial[((int64_t)m * sum_ctas + blockIdx.x) * kMaxLevels + l] = a[0];
         }
-    }
-    if (COUNTS) {
-        for (int l = 0; l < L; ++l) {
-            const uint32_t c = sh_cnt[l * kS2Threads + threadIdx.x];
-            if (c) atomicAdd(&sh_tot[l], c);
-        }
-        __syncthreads();
-        if (threadIdx.x < L) region_partial[((int64_t)m * sum_ctas + blockIdx.x) * kMaxLevels + threadIdx.x] = sh_tot[threadIdx.x];
     }
 }
 
@@ -947,9 +930,8 @@ static int cand_blocks(const Workspace& ws, int M) {
     return nb < 1 ? 1 : nb;
 }
 
-static size_t s2_smem(int L, bool sums, bool counts) {
-    return kBins1 + (size_t)kStage * 4 + (sums ? (size_t)L * kS2Threads * sizeof(double) : 0) +
-           (counts ? (size_t)L * kS2Threads * sizeof(uint32_t) : 0);
+static size_t s2_smem(int L, bool sums) {
+    return kBins1 + (size_t)kStage * 4 + (sums ? (size_t)L * kS2Threads * sizeof(double) : 0);
 }
 
 // Sweep 2: energies of the threshold-free bins (adaptive only) and the candidate keys of the boundary bins.
@@ -960,17 +942,17 @@ void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int6
     int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, sums ? 2 : 8);  // without the accumulators four blocks fit an SM
     if (nb > ws.sum_ctas) nb = ws.sum_ctas;
     ws.cur_sum_ctas = nb;
-    const size_t smem = s2_smem(L, sums, false);
+    const size_t smem = s2_smem(L, sums);
     LaunchScope t(ws, K_SUMS_CAND, s);
     if (sums)
-        sums_candidates_kernel<true, false><<<dim3(nb, M), kS2Threads, smem, s>>>(
-            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, nullptr, ws.sum_ctas, ws.cand_keys,
-            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr, ws.tile_max,
+        sums_candidates_kernel<true><<<dim3(nb, M), kS2Threads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys,
+            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, ws.tile_max,
             emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor);
     else
-        sums_candidates_kernel<false, false><<<dim3(nb, M), kS2Threads, smem, s>>>(
-            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, nullptr, ws.sum_ctas, ws.cand_keys,
-            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, nullptr, ws.tile_max,
+        sums_candidates_kernel<false><<<dim3(nb, M), kS2Threads, smem, s>>>(
+            static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys,
+            ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, ws.tile_max,
             emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor);
 }
 
@@ -1073,10 +1055,10 @@ int configure_select_kernels() {
     e = cudaFuncSetAttribute(norm_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxLevels * kSweepThreads * sizeof(double)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
-    const int smem_s2 = (int)s2_smem(kMaxLevels, true, false);  // 160 KB; with counts as well L is limited (see launcher)
-    e = cudaFuncSetAttribute(sums_candidates_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
+    const int smem_s2 = (int)s2_smem(kMaxLevels, true);
+    e = cudaFuncSetAttribute(sums_candidates_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
-    e = cudaFuncSetAttribute(sums_candidates_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
+    e = cudaFuncSetAttribute(sums_candidates_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_s2);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     e = cudaFuncSetAttribute(cand_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxLevels * 4 * kCandSumThreads * sizeof(unsigned long long)));
