@@ -272,6 +272,26 @@ def test_emission_reads_only_tiles_that_can_hold_band_entries(B, ctx, dtype):
                 assert listed[m] <= 4                       # the loud layer (two tiles, at most one more on each side)
 
 
+def test_many_workers_and_the_maximum_number_of_levels(B, ora):
+    """M = 700 workers with L = 32 levels (the largest the ABI takes), Top-k adaptive and fixed p, and bit-wise:
+    the per-worker tables of the emission and of the averaging kernels are sized by M."""
+    M, d = 700, 9_001
+    rng = np.random.default_rng(31)
+    g_np = (rng.standard_normal((M, d)) * 10.0 ** rng.uniform(-2, 0, (M, 1))).astype(np.float32)
+    g = to_dev(g_np)
+    c = B.mlmc_create(0, d, M, 32)
+    try:
+        k = sorted(set(int(x) for x in np.geomspace(1, d, 32)))
+        k += list(range(k[-1] - (32 - len(k)), k[-1]))      # pad with distinct values below d up to 32 levels
+        k = sorted(set(k))[-32:]
+        assert len(k) == 32 and k[-1] == d
+        check_topk(B, ora, c, g, k, None, 5, 0, expect_excluded=2)
+        check_topk(B, ora, c, g, k, list(wl.geometric_probs(32)), 5, 1, expect_excluded=2)
+        check_bitwise(B, ora, c, g, list(range(1, 24)), None, 5, 2)
+    finally:
+        B.mlmc_destroy(c)
+
+
 def test_level_probs(B, ora, ctx):
     w = wl.shrink(wl.C5A, 600_000, 4)
     k = wl.topk_schedule(w)
