@@ -510,7 +510,7 @@ BitSchedule make_schedule(const int32_t* b, int L) {
 int bit_blocks(const Workspace& ws, int64_t d, int vec, int M, int waves) {
     const int64_t nvec = (d + vec - 1) / vec;
     const int64_t by_work = (nvec + (int64_t)kSweepThreads * 4 - 1) / ((int64_t)kSweepThreads * 4);
-    int64_t by_sm = ((int64_t)ws.sm_count * waves + M - 1) / M;
+    int64_t by_sm = ((int64_t)ws.sm_count * waves) / M;  // rounded down: one block too many per worker costs a whole extra wave
     int64_t nb = by_work < by_sm ? by_work : by_sm;
     return (int)(nb < 1 ? 1 : nb);
 }
@@ -602,7 +602,7 @@ static void launch_bit_pack_t(Workspace& ws, const T* g, int64_t d, int M, int64
         w_low = sc.width[l] < w_low ? sc.width[l] : w_low;
     }
     if (w_low <= 8) {  // some level has a field of at most 8 bits
-        int64_t nb = ((int64_t)ws.sm_count * 3 + M - 1) / M;  // persistent: three resident blocks per SM
+        int64_t nb = ((int64_t)ws.sm_count * 3) / M;  // persistent: three resident blocks per SM, rounded down
         if (nb > by_work) nb = by_work;
         if (nb < 1) nb = 1;
         LaunchScope t(ws, K_BIT_PACK, s);
@@ -610,7 +610,7 @@ static void launch_bit_pack_t(Workspace& ws, const T* g, int64_t d, int M, int64
                                                                                 out.planes, out.w_max, words);
     }
     if (w_top > 8) {  // some level has a wider field
-        int64_t nb = ((int64_t)ws.sm_count * 2 + M - 1) / M;  // two resident blocks per SM
+        int64_t nb = ((int64_t)ws.sm_count * 2) / M;  // two resident blocks per SM, rounded down
         if (nb > by_work) nb = by_work;
         if (nb < 1) nb = 1;
         LaunchScope t(ws, K_BIT_PACK_WIDE, s);
@@ -633,7 +633,12 @@ void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const in
     const BitSchedule sc = make_schedule(b, L);
     const int64_t words = (d + 31) / 32;
     int64_t nb = (words + kBitThreads - 1) / kBitThreads;
-    const int64_t cap = (int64_t)ws.sm_count * 8;
+    // whole waves only: every block does the same number of iterations, so a partial last wave costs a full one
+    int resident = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, aggregate_bitwise_kernel, kBitThreads, 0) != cudaSuccess ||
+        resident < 1)
+        resident = 1;
+    const int64_t cap = (int64_t)ws.sm_count * resident * 2;
     if (nb > cap) nb = cap;
     LaunchScope t(ws, K_AGG_BIT, s);
     aggregate_bitwise_kernel<<<(unsigned)nb, kBitThreads, 0, s>>>(msgs.planes, msgs.gmax, msgs.level, msgs.p_sel, sc,

@@ -542,9 +542,20 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
                                                     ws.worker_tiles, ws.tile_n, ws.status);
     }
     const int wpb = kBandThreads / 32;
-    int64_t grid = (most + wpb - 1) / wpb;
-    if (grid > (int64_t)ws.sm_count * 8) grid = (int64_t)ws.sm_count * 8;
     const size_t smem = (size_t)(M + 1) * sizeof(uint32_t);
+    const size_t smem_w = smem + (size_t)(kBandThreads / 32) * kWriteSlots * kBatchWords * sizeof(uint32_t);
+    // grids of two whole waves: the warps take tiles with a grid stride, so a partial last wave costs a full one
+    auto two_waves = [&](const void* kernel, size_t dyn_smem) -> int64_t {
+        int resident = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kBandThreads, dyn_smem) != cudaSuccess || resident < 1)
+            resident = 1;
+        int64_t grid = (int64_t)ws.sm_count * resident * 2;
+        const int64_t by_work = (most + wpb - 1) / wpb;
+        return grid < by_work ? grid : by_work;
+    };
+    const bool bf = dtype == MLMC_BF16;
+    const int64_t grid = two_waves(bf ? (const void*)band_count_kernel<bf16_t> : (const void*)band_count_kernel<float>, smem);
+    const int64_t grid_w = two_waves(bf ? (const void*)band_write_kernel<bf16_t> : (const void*)band_write_kernel<float>, smem_w);
     {
         LaunchScope t(ws, K_BAND_COUNT, s);
         if (dtype == MLMC_BF16)
@@ -559,13 +570,12 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
         band_scan_kernel<<<M, kListThreads, 0, s>>>(ws.tile_desc, tpw, ws.tile_n, ws.emit, ws.status);
     }
     LaunchScope t(ws, K_EMIT, s);
-    const size_t smem_w = smem + (size_t)(kBandThreads / 32) * kWriteSlots * kBatchWords * sizeof(uint32_t);
     if (dtype == MLMC_BF16)
-        band_write_kernel<bf16_t><<<(unsigned)grid, kBandThreads, smem_w, s>>>(
+        band_write_kernel<bf16_t><<<(unsigned)grid_w, kBandThreads, smem_w, s>>>(
             static_cast<const bf16_t*>(g), d, ld, tpw, ws.worker_tiles, ws.tile_n, M, ws.emit, ws.tile_desc, out.idx,
             out.val, out.capacity);
     else
-        band_write_kernel<float><<<(unsigned)grid, kBandThreads, smem_w, s>>>(
+        band_write_kernel<float><<<(unsigned)grid_w, kBandThreads, smem_w, s>>>(
             static_cast<const float*>(g), d, ld, tpw, ws.worker_tiles, ws.tile_n, M, ws.emit, ws.tile_desc, out.idx,
             out.val, out.capacity);
 }

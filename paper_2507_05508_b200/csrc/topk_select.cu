@@ -868,7 +868,7 @@ __global__ void copy_probs_kernel(const double* p_all, const double* delta_all, 
 int blocks_per_worker(const Workspace& ws, int64_t d, int vec, int threads, int M, int waves) {
     const int64_t nvec = (d + vec - 1) / vec;
     const int64_t by_work = (nvec + (int64_t)threads * 4 - 1) / ((int64_t)threads * 4);
-    int64_t by_sm = ((int64_t)ws.sm_count * waves + M - 1) / M;
+    int64_t by_sm = ((int64_t)ws.sm_count * waves) / M;  // rounded down: one block too many per worker costs a whole extra wave
     if (by_sm < 1) by_sm = 1;
     int64_t nb = by_work < by_sm ? by_work : by_sm;
     return (int)(nb < 1 ? 1 : nb);
@@ -926,7 +926,7 @@ void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
 }
 
 static int cand_blocks(const Workspace& ws, int M) {
-    int nb = (ws.sm_count * 2 + M - 1) / M;
+    int nb = (ws.sm_count * 2) / M;
     return nb < 1 ? 1 : nb;
 }
 
