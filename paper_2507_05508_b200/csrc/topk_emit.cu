@@ -395,8 +395,63 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
                 uint32_t tA = rA, tB = rB;  // tie ranks, advanced row by row on the ties path
                 const uint32_t e0 = (uint32_t)((tile * kEmitTile + (int64_t)b * kBatchWords + lane) * S);
                 uint32_t rows = (rowany | (rowany >> 16)) & 0xFFFFu;  // rows that hold a closed-range key
-                // a rolled loop over the rows that matter: the body is long, unrolling it 16 times would not fit the
-                // instruction cache
+                if (!ties) {
+                    // No tie needs ranking: membership follows from the entry's own key.  Two rows per trip, so that
+                    // the ballots and counts of one row do not wait for the position arithmetic of the other.
+                    auto member = [&](uint32_t w, int i, int s) -> bool {
+                        bool em = (flags >> (i + 16 * s)) & 1u;
+                        if (drop_any) {  // warp-uniform
+                            const uint32_t tk = EW::key(w, s) - Tb;
+                            em = em && !(dropA && tk == W) && !(dropB && tk == 0u);
+                        }
+                        return em;
+                    };
+#pragma unroll 1
+                    while (rows) {
+                        constexpr int R = 2;  // rows per trip (four need 74 registers and lose a resident block)
+                        int ri[R];
+                        bool on[R];  // warp-uniform
+                        uint32_t wv[R];
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            on[r] = rows != 0u;
+                            ri[r] = on[r] ? __ffs(rows) - 1 : 0;
+                            if (on[r]) rows &= rows - 1u;
+                            wv[r] = slot[ri[r] * 32];
+                        }
+                        bool em[R][S];
+                        uint32_t below[R], cnt[R];
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            below[r] = 0;
+                            cnt[r] = 0;
+#pragma unroll
+                            for (int s = 0; s < S; ++s) {
+                                em[r][s] = on[r] && member(wv[r], ri[r], s);
+                                const uint32_t mk = __ballot_sync(0xFFFFFFFFu, em[r][s]);
+                                below[r] += __popc(mk & lt);
+                                cnt[r] += __popc(mk);
+                            }
+                        }
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            uint32_t pos = base + below[r];
+                            base += cnt[r];  // the base of the next row
+#pragma unroll
+                            for (int s = 0; s < S; ++s) {
+                                if (em[r][s]) {
+                                    if ((int64_t)pos < capacity) {
+                                        idx_w[pos] = e0 + (uint32_t)(ri[r] * 32 * S + s);
+                                        val_w[pos] = EW::value(wv[r], s) * inv_p;
+                                    }
+                                    ++pos;
+                                }
+                            }
+                        }
+                    }
+                }
+                // ties to rank: a rolled loop over the rows that matter, each row continuing from the one before
+                // (the body is long, unrolling it 16 times would not fit the instruction cache)
 #pragma unroll 1
                 while (rows) {
                     const int i = __ffs(rows) - 1;
