@@ -90,6 +90,7 @@ int finish(cudaError_t e) { return e == cudaSuccess ? MLMC_OK : MLMC_ERR_CUDA; }
 // digit passes over the candidates.
 void run_selection(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, int L, bool sums,
                    cudaStream_t s) {
+    launch_reset_selection(ws, dtype, d, M, s);
     launch_hist1(ws, g, dtype, d, M, ld, s);
     launch_resolve1(ws, dtype, M, L, s);
     if (dtype == MLMC_F32) {
@@ -270,7 +271,7 @@ int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches :
 static const char* const kKernelNames[K_COUNT] = {
     "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "sums_candidates", "cand_pass2", "masked_pass2",
     "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
-    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide"};
+    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide", "reset"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
 

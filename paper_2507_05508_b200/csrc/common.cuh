@@ -51,7 +51,7 @@ struct EmitParams {
 enum KernelId {
     K_DRAW_FIXED = 0, K_INIT_QUERIES, K_UNIFORMS, K_HIST1, K_RESOLVE1, K_SUMS_CAND, K_CAND2, K_MASKED2, K_RESOLVE2, K_CAND3,
     K_MASKED3, K_RESOLVE3, K_CAND_SUMS, K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
-    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_TILE_LIST, K_BAND_COUNT, K_BAND_SCAN, K_BIT_PACK_WIDE, K_COUNT
+    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_TILE_LIST, K_BAND_COUNT, K_BAND_SCAN, K_BIT_PACK_WIDE, K_RESET, K_COUNT
 };
 
 constexpr int kTimingPool = 2048;  // event pairs kept between two reads
@@ -240,6 +240,7 @@ int configure_select_kernels();
 void launch_init_queries_adaptive(Workspace& ws, int M, int L, int64_t d, cudaStream_t s);
 void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, cudaStream_t s);
 void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStream_t s);
+void launch_reset_selection(Workspace& ws, int dtype, int64_t d, int M, cudaStream_t s);
 void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s);
 void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s);
 void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,

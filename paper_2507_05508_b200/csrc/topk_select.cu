@@ -865,6 +865,25 @@ __global__ void copy_probs_kernel(const double* p_all, const double* delta_all, 
     if (delta_out) delta_out[i] = bad ? 0.0 : delta_all[m * kMaxLevels + l];
 }
 
+// Everything a selection accumulates into, cleared by one launch: the three histograms, the tile maxima, the
+// candidate counters and sums (zero), and the digit-2 slot map ("no slot").
+struct ResetList {
+    uint32_t* ptr[8];
+    uint32_t words[8];
+    uint32_t value[8];
+    int n;
+};
+
+__global__ void reset_state_kernel(ResetList r) {
+    for (int a = 0; a < r.n; ++a) {
+        uint32_t* p = r.ptr[a];
+        const uint32_t n4 = r.words[a] / 4, v = r.value[a];
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x)
+            reinterpret_cast<uint4*>(p)[i] = make_uint4(v, v, v, v);
+        for (uint32_t i = n4 * 4 + blockIdx.x * blockDim.x + threadIdx.x; i < r.words[a]; i += gridDim.x * blockDim.x) p[i] = v;
+    }
+}
+
 int blocks_per_worker(const Workspace& ws, int64_t d, int vec, int threads, int M, int waves) {
     const int64_t nvec = (d + vec - 1) / vec;
     const int64_t by_work = (nvec + (int64_t)threads * 4 - 1) / ((int64_t)threads * 4);
@@ -902,10 +921,32 @@ void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStr
     uniforms_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.u_dev, M, seed, step);
 }
 
+// One launch instead of nine memsets, before the first sweep.
+void launch_reset_selection(Workspace& ws, int dtype, int64_t d, int M, cudaStream_t s) {
+    const int tpw = emit_tiles_per_worker(d, dtype);
+    ResetList r = {};
+    auto add = [&](void* p, size_t bytes, uint32_t value) {
+        r.ptr[r.n] = static_cast<uint32_t*>(p);
+        r.words[r.n] = (uint32_t)(bytes / 4);
+        r.value[r.n] = value;
+        ++r.n;
+    };
+    add(ws.hist1, (size_t)M * kBins1 * sizeof(uint32_t), 0u);
+    add(ws.tile_max, (size_t)M * tpw * sizeof(uint32_t), 0u);
+    if (dtype == MLMC_F32) {
+        add(ws.cand_count, sizeof(uint32_t) * M, 0u);
+        add(ws.cand_overflow, sizeof(int) * M, 0u);
+        add(ws.hist2, (size_t)M * kMaxQueries * kBins23 * sizeof(uint32_t), 0u);
+        add(ws.map2, (size_t)M * kMaxQueries * kBins23, 0xFFFFFFFFu);
+        add(ws.hist3, (size_t)M * kMaxQueries * kBins23 * sizeof(uint32_t), 0u);
+        add(ws.cand_S, (size_t)M * kMaxLevels * 4 * sizeof(unsigned long long), 0u);
+    }
+    LaunchScope t(ws, K_RESET, s);
+    reset_state_kernel<<<ws.sm_count * 2, 512, 0, s>>>(r);
+}
+
 void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
     const int tpw = emit_tiles_per_worker(d, dtype);
-    cudaMemsetAsync(ws.hist1, 0, (size_t)M * kBins1 * sizeof(uint32_t), s);
-    cudaMemsetAsync(ws.tile_max, 0, (size_t)M * tpw * sizeof(uint32_t), s);
     const size_t smem = kBins1 * sizeof(uint32_t);
     LaunchScope t(ws, K_HIST1, s);
     if (dtype == MLMC_BF16) {
@@ -937,8 +978,6 @@ static size_t s2_smem(int L, bool sums) {
 // Sweep 2: energies of the threshold-free bins (adaptive only) and the candidate keys of the boundary bins.
 void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,
                             cudaStream_t s) {
-    cudaMemsetAsync(ws.cand_count, 0, sizeof(uint32_t) * M, s);
-    cudaMemsetAsync(ws.cand_overflow, 0, sizeof(int) * M, s);
     int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, sums ? 2 : 8);  // without the accumulators four blocks fit an SM
     if (nb > ws.sum_ctas) nb = ws.sum_ctas;
     ws.cur_sum_ctas = nb;
@@ -958,13 +997,10 @@ void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int6
 
 // Digit pass 2 or 3: over the candidate keys, and (early exit unless the buffer overflowed) over the full row.
 void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s) {
-    const size_t hist_bytes = (size_t)M * kMaxQueries * kBins23 * sizeof(uint32_t);
     const size_t smem = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
     const int nb_full = blocks_per_worker(ws, d, 4, kSweepThreads, M, 2);  // fall-back sweeps: a small grid, since they normally exit at once
     const int nb_cand = cand_blocks(ws, M);
     if (pass == 2) {
-        cudaMemsetAsync(ws.hist2, 0, hist_bytes, s);
-        cudaMemsetAsync(ws.map2, 0xFF, (size_t)M * kMaxQueries * kBins23, s);
         {
             LaunchScope t(ws, K_CAND2, s);
             cand_pass_kernel<2><<<dim3(nb_cand, M), kSweepThreads, 0, s>>>(ws.cand_keys, ws.cand_cap, ws.cand_count,
@@ -975,7 +1011,6 @@ void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t l
         masked_pass_kernel<2><<<dim3(nb_full, M), kSweepThreads, smem, s>>>(
             static_cast<const float*>(g), d, ld, ws.table1, ws.map2, ws.hist2, ws.worker_err, ws.cand_overflow);
     } else {
-        cudaMemsetAsync(ws.hist3, 0, hist_bytes, s);
         {
             LaunchScope t(ws, K_CAND3, s);
             cand_pass_kernel<3><<<dim3(nb_cand, M), kSweepThreads, 0, s>>>(ws.cand_keys, ws.cand_cap, ws.cand_count,
@@ -1000,7 +1035,6 @@ void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
 void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s) {
     {
         const int nb = 3 * cand_blocks(ws, M);
-        cudaMemsetAsync(ws.cand_S, 0, (size_t)M * kMaxLevels * 4 * sizeof(unsigned long long), s);
         LaunchScope t(ws, K_CAND_SUMS, s);
         cand_sums_kernel<<<dim3(nb, M), kCandSumThreads, (size_t)L * 4 * kCandSumThreads * sizeof(unsigned long long), s>>>(
             ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.queries, L, ws.cand_S, ws.worker_err);
