@@ -14,8 +14,8 @@
  *  - Pointers are DEVICE pointers unless marked "host".  The caller owns every buffer; the library
  *    only owns the scratch workspace inside mlmc_ctx.
  *  - All work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default
- *    stream).  Nothing synchronises except mlmc_create, mlmc_destroy, mlmc_get_status, mlmc_read_u and
- *    mlmc_read_listed_tiles.
+ *    stream).  Nothing synchronises except mlmc_create, mlmc_destroy and mlmc_get_status (and the
+ *    measurement calls of mlmc_instr.h, which are not part of the method).
  *  - The int return value reports host-side checks made before any launch (arguments, schedule,
  *    probabilities).  Conditions found on the device (message capacity, non-finite input, a bounded
  *    wait that gave up) are written to a sticky status word read by mlmc_get_status; the affected
@@ -89,31 +89,6 @@ int mlmc_destroy(mlmc_ctx* ctx);
 /* Synchronises `stream`, returns the sticky device status (first error since the last call) and clears it. */
 int mlmc_get_status(mlmc_ctx* ctx, void* stream);
 
-/* Number of kernels this ctx has launched so far (host counter; for launch accounting). */
-int64_t mlmc_launch_count(const mlmc_ctx* ctx);
-
-/* Per-kernel timing for roofline measurements (instrumentation of this library; not part of the
- * method).  With timing on, every kernel launch is bracketed by a CUDA event pair on its stream (at
- * most 2048 launches between two reads; later ones are not recorded).  mlmc_timing_read synchronises
- * `stream`, fills total_ms[id] and launches[id] for id < mlmc_kernel_count() (host arrays) with the
- * launches recorded since the previous read, and restarts the record. */
-int mlmc_kernel_count(void);
-const char* mlmc_kernel_name(int id);
-int mlmc_timing_enable(mlmc_ctx* ctx, int on);
-int mlmc_timing_read(mlmc_ctx* ctx, double* total_ms, int64_t* launches, void* stream);
-
-/* The uniforms of the level draw for workers 0..M-1 at (seed, step), computed on the device and
- * copied to u_host[M].  Synchronous; for checking the counter generator against known answers. */
-int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream);
-
-/* How much of every row the last mlmc_compress_topk on this context read when it emitted the bands (the
- * band of ranks (k_{l-1}, k_l] of Sec. 3.2): the emission reads only the tiles of 4096 32-bit words (4096 fp32
- * or 8192 bf16 entries) whose largest magnitude reaches the band's lower threshold, twice each.
- *   listed_host  host uint32 [M]: tiles of worker m that were read.
- *   tiles_host   host int64: tiles in one row.
- * Synchronous (copies from the device and waits for the stream); a measurement aid, not part of the method. */
-int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t* tiles_host, void* stream);
-
 /* Level probabilities and residual norms (Lemma 3.4; Alg. 3 "Compute p^l = Delta^l / sum Delta").
  *   kind   MLMC_TOPK: sched = host int64 k[L];  MLMC_BITWISE: sched = host int64 b[L].
  *   p_host NULL: adaptive, p_out[m][l] = Delta_l / sum Delta (all weight on level 0 if every Delta is 0).
@@ -164,7 +139,9 @@ int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, 
  *   Limit       M * (ceil(d / 4096) + 1) <= 2^20; larger problems return MLMC_ERR_ARG and nothing is launched.
  *   Device      the current device of the calling thread; msgs and out must live there.
  *   First call  on each device looks up the device address of the built-in table (a synchronous
- *               runtime query); make that first call before starting any stream capture.
+ *               runtime query); make that first call before starting any stream capture.  Host threads
+ *               may make their first calls on a device concurrently: the looked-up values are published
+ *               with release/acquire ordering and looking them up twice is harmless.
  *   Sharing     every call on a device uses the same table.  Each call rewrites all entries it reads,
  *               so nothing carries over between calls, but two calls whose kernels overlap on the GPU
  *               (different streams, or several host threads) race: run them one after the other.

@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "../../include/mlmc.h"
+#include "../../include/mlmc_instr.h"
 
 namespace mlmc {
 

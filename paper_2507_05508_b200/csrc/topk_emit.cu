@@ -15,6 +15,8 @@
 // aggregate: the dense mean (1/M) sum_m g~_m (Alg. 2 "Server aggregates") tiled over the index
 // space; because every message is index-sorted, a tile's entries are one contiguous range per
 // worker; they are added into a shared-memory tile in worker order and the tile is written once.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace mlmc {
@@ -665,7 +667,11 @@ constexpr int64_t kStaticOffsetWords = int64_t(1) << 20;  // 4 MiB: M * (ceil(d 
 static __device__ __align__(256) uint32_t g_static_offsets[kStaticOffsetWords];
 
 constexpr int kMaxDevices = 64;
-uint32_t* g_static_offsets_addr[kMaxDevices];  // device address of the array on each device, 0 = not looked up yet
+// Device address of the array on each device, 0 = not looked up yet.  Host threads may make their first call on a
+// device at the same time: the SM count is written first and the address is published last with a release store,
+// so a thread that sees the address (acquire load) also sees the count.  Two threads that both find 0 look the
+// same values up twice, which is harmless.
+std::atomic<uint32_t*> g_static_offsets_addr[kMaxDevices];
 int g_static_sm_count[kMaxDevices];
 
 }  // namespace
@@ -680,7 +686,8 @@ extern "C" int mlmc_aggregate_topk_noalloc(const mlmc_topk_msgs* msgs, int M, in
     if (n_off > kStaticOffsetWords) return MLMC_ERR_ARG;  // beyond the fixed scratch: use mlmc_aggregate with a context
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MLMC_ERR_CUDA;
-    if (!g_static_offsets_addr[dev]) {
+    uint32_t* offsets = g_static_offsets_addr[dev].load(std::memory_order_acquire);
+    if (!offsets) {
         // Set-up, once per device, with that device current.  In host code the array's name only stands
         // for the symbol; the address a kernel can use has to be asked for.
         uint32_t* p = nullptr;
@@ -692,9 +699,9 @@ extern "C" int mlmc_aggregate_topk_noalloc(const mlmc_topk_msgs* msgs, int M, in
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
             return MLMC_ERR_CUDA;
         g_static_sm_count[dev] = sms;
-        g_static_offsets_addr[dev] = p;
+        g_static_offsets_addr[dev].store(p, std::memory_order_release);
+        offsets = p;
     }
-    uint32_t* offsets = g_static_offsets_addr[dev];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // every entry in [0, n_off) is rewritten by this kernel, so nothing is left over from an earlier call
     agg_offsets_kernel<<<(unsigned)((n_off + 255) / 256), 256, 0, s>>>(msgs->idx, msgs->count, msgs->level,

@@ -589,9 +589,10 @@ resolve23_kernel(const uint32_t* hist, Query* queries, uint8_t* map2, int nq, co
             cnt[i] = h[255 - (lane * 8 + i)];
             local += cnt[i];
         }
+        const uint32_t rem = qq.rem, prefix = qq.prefix;  // read by every lane before the owning lane rewrites them
         const uint32_t inc = warp_inclusive_sum(local);
-        const uint32_t rem = qq.rem;
         const bool mine = (inc >= rem) && (inc - local < rem);
+        __syncwarp();
         if (mine) {
             uint32_t above = inc - local;
 #pragma unroll
@@ -599,10 +600,10 @@ resolve23_kernel(const uint32_t* hist, Query* queries, uint8_t* map2, int nq, co
                 if (above + cnt[i] >= rem) {
                     const uint32_t digit = 255u - (uint32_t)(lane * 8 + i);
                     if (PASS == 2) {
-                        qq.prefix |= digit << 8;
+                        qq.prefix = prefix | (digit << 8);
                         qq.rem = rem - above;
                     } else {
-                        qq.T = qq.prefix | digit;
+                        qq.T = prefix | digit;
                         qq.r = rem - above;
                         qq.n = cnt[i];
                         qq.c = qq.k - qq.r;

@@ -1,4 +1,4 @@
-"""CPU-side checks: the C-ABI library loads and exports what include/mlmc.h declares; workload generators."""
+"""CPU-side checks: the C-ABI library loads and exports what include/*.h declare; workload generators."""
 import ctypes
 import os
 import re
@@ -11,7 +11,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "mlmc.h")).read()
+    inc = os.path.join(ROOT, "include")
+    text = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(mlmc_[a-z_0-9]+)\s*\(", text)))
 

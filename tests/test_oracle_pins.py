@@ -413,6 +413,39 @@ def test_aggregate_topk(ora):
     assert np.allclose(out2, out, rtol=1e-15, atol=0)
 
 
+def test_aggregate_scale_is_the_mean_of_absolute_terms_hand_example(ora):
+    """Alg. 2 "Server aggregates" on hand-written messages: M = 3 workers, overlapping coordinates, mixed signs.
+    The expected mean and the expected tolerance scale (1/M) sum_m |term_m| are typed in by hand (exact in binary)."""
+    d = 6
+    msgs = [(np.array([0, 2, 5], dtype=np.uint32), np.array([1.5, -3.0, 0.75], dtype=np.float32)),
+            (np.array([2, 3], dtype=np.uint32), np.array([3.0, -6.0], dtype=np.float32)),
+            (np.array([0, 2, 3], dtype=np.uint32), np.array([-4.5, 1.5, -1.5], dtype=np.float32))]
+    out, scale = ora.aggregate_topk(msgs, d)
+    assert out.tolist() == [-1.0, 0.0, 0.5, -2.5, 0.0, 0.25]
+    assert scale.tolist() == [2.0, 0.0, 2.5, 2.5, 0.0, 0.25]
+    # the scale is a mean, not a sum: the same three messages sent twice (M = 6) leave it unchanged
+    out6, scale6 = ora.aggregate_topk(msgs + msgs, d)
+    assert out6.tolist() == out.tolist() and scale6.tolist() == scale.tolist()
+
+
+def test_aggregate_bitwise_scale_hand_example(ora):
+    """Bit-plane messages typed in by hand: b = (1, 3), d = 3, M = 2.  Worker 0 sends level 1 (a 2-bit field) with
+    gmax 4 and p 1/2, worker 1 sends level 0 (a 1-bit field) with gmax 2 and p 1/4.  A residual entry is
+    sign f 2^-b_l gmax / p (Sec. 3.1), so the terms are (3, -1, 0) and (-4, 0, 4); mean and scale follow by hand."""
+    class Msg:
+        pass
+    a, c = Msg(), Msg()
+    # worker 0: fields (3, 1, 0) -> planes: sign 0b010, msb 0b001, lsb 0b011; unit = 2^-3 * 4 / (1/2) = 1
+    a.planes = np.array([[0b010], [0b001], [0b011]], dtype=np.uint32)
+    a.gmax, a.level, a.p_sel = 4.0, 1, 0.5
+    # worker 1: fields (1, 0, 1) -> planes: sign 0b001, bit 0b101; unit = 2^-1 * 2 / (1/4) = 4
+    c.planes = np.array([[0b001], [0b101]], dtype=np.uint32)
+    c.gmax, c.level, c.p_sel = 2.0, 0, 0.25
+    out, scale = ora.aggregate_bitwise([a, c], [1, 3], 3)
+    assert out.tolist() == [-0.5, -0.5, 2.0]
+    assert scale.tolist() == [3.5, 0.5, 2.0]
+
+
 def test_aggregate_bitwise(ora):
     rng = np.random.default_rng(15)
     d, M = 130, 4

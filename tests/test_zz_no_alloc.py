@@ -4,8 +4,10 @@ Some callers cannot create an mlmc_ctx because that calls cudaMalloc: a serving 
 framework has already taken the whole GPU for its pool, or code running where the allocator must not
 be entered.  mlmc_aggregate_topk_noalloc serves them from a scratch table built into the library.
 It launches the same kernels as mlmc_aggregate, so the two results must agree bit for bit; the check
-runs on two calls in a row with different messages, since every call reuses the same table.
+runs on two calls in a row with different messages, since every call reuses the same table.  The result
+is also held against the CPU oracle's fp64 average of the same messages (Alg. 2, "Server aggregates").
 """
+import numpy as np
 import pytest
 import torch
 
@@ -14,7 +16,7 @@ from paper_2507_05508_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-def test_noalloc_aggregate_matches_context_aggregate_twice():
+def test_noalloc_aggregate_matches_context_aggregate_twice(ora):
     from paper_2507_05508_b200 import binding as B
     B.lib()
     torch.cuda.set_device(0)
@@ -36,6 +38,11 @@ def test_noalloc_aggregate_matches_context_aggregate_twice():
             torch.cuda.synchronize()
             assert not torch.isnan(got).any()
             assert torch.equal(got, ref)             # same kernels, same order of additions: tolerance 0 <= 1e-6
+            n = msgs.count.tolist()
+            host = [(msgs.idx[m, :n[m]].cpu().numpy().view(np.uint32), msgs.val[m, :n[m]].cpu().numpy())
+                    for m in range(w.M)]
+            mean, scale = ora.aggregate_topk(host, w.d)
+            assert np.all(np.abs(got.cpu().numpy().astype(np.float64) - mean) <= 1e-6 * scale + 1e-45)
         # beyond the built-in table (M * (tiles + 1) > 2^20): refused with an argument error, nothing is launched
         import ctypes
         rc = B.lib().mlmc_aggregate_topk_noalloc(ctypes.byref(msgs.struct), 1, (1 << 32) - 1, got.data_ptr(), None)
