@@ -8,7 +8,8 @@ synthetic gradients already resident in HBM.  The default workload c5 is the 124
 both of its variants per step (adaptive MLMC-Top-k, then adaptive bit-wise MLMC, each a full
 compress + aggregate over the same gradient batch).  `value` is gradient GB/s = gradient bytes swept by
 the variants (M*d*sizeof(T) each) / step time, summed over ranks (ranks are independent replicas: the
-path has no inter-GPU exchange).
+path has no inter-GPU exchange).  On one GPU the default run also times c4, c5a, c5b and c3 for a few steps each
+and reports them under `also` in the same line.
 Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
@@ -29,14 +30,22 @@ METRIC = "MLMC compress+aggregate gradient GB/s per step (1 B200); fraction of H
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic per launch of each sweep kernel relative to its algorithmic bytes, from the ncu captures
-# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same
-# kernel; traffic grows in proportion to the elements swept).  None = not captured yet.
-NCU_TRAFFIC_RATIO = {
-    # profiles/c5_small_kernels.md (fp32, d = 32e6, M = 4).  band_count and emit read only the listed tiles, a share
-    # of the row that changes with the drawn levels: no fixed ratio, their traffic is reported as null.
-    "hist1:f32": 1.008, "sums_candidates:f32": 1.010, "absmax:f32": 1.007, "bit_stats:f32": 1.008, "bit_pack:f32": 1.00,
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic_ratios.txt")
+
+
+def ncu_traffic_ratios():
+    """DRAM traffic per launch of a sweep kernel relative to its algorithmic bytes, from the ncu captures summarised
+    under profiles/ (one line per kernel: `kernel:dtype ratio`).  A kernel that has no line, or whose line was
+    removed because the kernel changed after the capture, reports traffic null."""
+    out = {}
+    try:
+        for ln in open(TRAFFIC_FILE):
+            ln = ln.split("#")[0].split()
+            if len(ln) == 2:
+                out[ln[0]] = float(ln[1])
+    except OSError:
+        pass
+    return out
 
 
 def parse_args():
@@ -48,6 +57,8 @@ def parse_args():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true", help="skip the shorter runs of c4, c5a, c5b and c3 reported under `also`")
+    ap.add_argument("--also-steps", type=int, default=10)
     ap.add_argument("--shrink-d", type=int, default=0, help="profiling aid: same workload structure at a smaller d")
     ap.add_argument("--shrink-M", type=int, default=0)
     return ap.parse_args()
@@ -233,101 +244,136 @@ def sweeps_charged(w, emit_read_frac=None) -> float:
     return 3.0 if w.adaptive else 2.0
 
 
-# Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes of its variant, dense bytes).
-# band_count and emit read only the tiles that can hold band entries (a fraction of the row that depends on the
-# drawn levels); they are charged a whole sweep here, so their figure can exceed the copy peak when few tiles are listed.
-def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float):
+# Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes of its variant, dense
+# bytes, share of the row in the listed tiles).  band_count and emit read only the tiles that can hold band entries,
+# so they are charged that share of the row; the candidate sweep of fixed p also skips tiles, by a share that is not
+# read back, so its bytes are unknown (None) there.
+def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float, read_frac, adaptive: bool):
     mt, mb = msg.get("topk", 0.0), msg.get("bitwise", 0.0)
+    listed = None if read_frac is None else read_frac * sweep
     table = {
-        "hist1": sweep, "sums_candidates": sweep, "masked_pass2": sweep, "masked_pass3": sweep, "norm_sweep": sweep,
-        "band_count": sweep, "emit": sweep + mt, "aggregate_topk": mt + dense,
+        "hist1": sweep, "sums_candidates": sweep if adaptive else None, "masked_pass2": sweep, "masked_pass3": sweep,
+        "norm_sweep": sweep, "band_count": listed, "emit": None if listed is None else listed + mt,
+        "aggregate_topk": mt + dense,
         "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + mb, "aggregate_bitwise": mb + dense,
     }
     return table.get(name)
 
 
-def run_cuda(args):
+def l2_policy(sweep_bytes: float, n_batches: int) -> str:
+    l2 = 126e6
+    if sweep_bytes > l2:
+        return f"inputs larger than L2: {sweep_bytes / 1e6:.0f} MB per sweep, {n_batches} batches alternated"
+    return (f"inputs smaller than L2 ({sweep_bytes / 1e6:.1f} MB per sweep): a {2 * l2 / 1e6:.0f} MB buffer is written "
+            "between timed steps (flush), outside the event pairs")
+
+
+def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, peak: float, peak_kind: str,
+            e2e_steps: int = 0):
+    """Times `steps` steps of one workload on this rank's GPU and returns its figures.  Three loops: the headline
+    loop (device-timed, nothing else enqueued), a second loop with one CUDA event pair around every kernel launch
+    (per-kernel times, message volume and the share of the row the emission read, step by step), and optionally
+    the end-to-end loop with host buffers."""
     import torch
-    from paper_2507_05508_b200 import build as cuda_build
-    from paper_2507_05508_b200 import workloads as wl
-    cuda_build.build()
-    rank, world, local = dist_setup(args.gpus)
-    subs = sub_workloads(args.workload)
-    if args.shrink_d or args.shrink_M:
-        subs = [wl.shrink(x, args.shrink_d or x.d, args.shrink_M or x.M) for x in subs]
     w = subs[0]
-    peak, peak_kind = measured_peak()
     r = Runner(subs, local, rank=rank)
     B = r.B
     sweep_bytes = float(w.M) * w.d * elem_size(w)
     dense_bytes = float(w.d) * 4.0
+    small = sweep_bytes <= 126e6
+    flush = torch.empty(int(252e6) // 4, dtype=torch.float32, device=r.dev) if small else None
 
-    for i in range(max(args.warmup, 3)):
+    for i in range(max(warmup, 3)):
         r.step(i)
     torch.cuda.synchronize()
     assert B.mlmc_get_status(r.ctx) == 0, "device status after warm-up"
 
-    # ---- timed region: exactly K steps, device-timed, per-kernel event pairs on the same stream
-    B.mlmc_timing_enable(r.ctx, True)
+    # ---- headline loop: exactly `steps` steps, device-timed, per-kernel timing off
     launches0 = B.mlmc_launch_count(r.ctx)
-    msg_acc = {}
     sampler = ClockSampler(local)
     barrier(world)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_wall0 = time.time()
-    e0.record()
-    for i in range(args.steps):
-        r.step(args.warmup + i)
-    e1.record()
-    torch.cuda.synchronize()
+    if small:  # an L2-sized input: flush between steps, every step has its own event pair
+        local_ms = 0.0
+        for i in range(steps):
+            flush.fill_(float(i))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            r.step(warmup + i)
+            e1.record()
+            torch.cuda.synchronize()
+            local_ms += e0.elapsed_time(e1)
+    else:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            r.step(warmup + i)
+        e1.record()
+        torch.cuda.synchronize()
+        local_ms = e0.elapsed_time(e1)
     barrier(world)
     t_wall = time.time() - t_wall0
     clocks = sampler.stop()
-    local_ms = e0.elapsed_time(e1)
     total_ms = max_over_ranks(local_ms, world, r.dev)
     launches = B.mlmc_launch_count(r.ctx) - launches0
-    per_kernel = B.mlmc_timing_read(r.ctx)
-    B.mlmc_timing_enable(r.ctx, False)
     status = B.mlmc_get_status(r.ctx)
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     value = world * len(subs) * sweep_bytes / (ms_per_step * 1e-3) / 1e9
 
-    # message volume: average over a few steps outside the timed region (levels are redrawn every step)
-    probe = min(args.steps, 8)
+    # ---- second loop, same steps: per-kernel event pairs, message volume, listed tiles (read back after every step)
+    B.mlmc_timing_enable(r.ctx, True)
+    per_kernel, msg_acc = {}, {}
     listed_acc, listed_n = 0.0, 0
+    probe = min(steps, 16)
     for i in range(probe):
-        r.step(args.warmup + i)
+        if small:
+            flush.fill_(float(i))
+        r.step(warmup + i)
+        for name, (ms, n) in B.mlmc_timing_read(r.ctx).items():
+            acc = per_kernel.setdefault(name, [0.0, 0])
+            acc[0] += ms
+            acc[1] += n
         for kind, v in r.message_bytes().items():
             msg_acc[kind] = msg_acc.get(kind, 0.0) + v
         if any(x.kind == "topk" for x in subs):
             listed, tiles = B.mlmc_read_listed_tiles(r.ctx, w.M)
             listed_acc += sum(listed) / float(max(1, tiles * w.M))
             listed_n += 1
+    B.mlmc_timing_enable(r.ctx, False)
     emit_read_frac = (listed_acc / listed_n) if listed_n else None
     msg_by_kind = {kind: v / probe for kind, v in msg_acc.items()}
     msg_bytes = sum(msg_by_kind.values())
 
     # ---- roofline of the dominant kernel and of the whole step
-    dom = max(per_kernel.items(), key=lambda kv: kv[1][0])
-    dom_name, (dom_ms, dom_n) = dom
-    dom_bytes = kernel_alg_bytes(dom_name, sweep_bytes, msg_by_kind, dense_bytes) or sweep_bytes
+    ratios = ncu_traffic_ratios()
+    adaptive_topk = any(x.kind == "topk" and x.adaptive for x in subs)
+    kernels = {}
+    t_all = sum(v[0] for v in per_kernel.values())
+    for name, (ms, n) in sorted(per_kernel.items(), key=lambda kv: -kv[1][0]):
+        kb = kernel_alg_bytes(name, sweep_bytes, msg_by_kind, dense_bytes, emit_read_frac, adaptive_topk)
+        avg_ms = ms / n
+        ach = None if not kb else kb / (avg_ms * 1e-3) / 1e9
+        kernels[name] = {"ms_per_step": round(ms / probe, 4), "launches_per_step": n / probe,
+                         "share": round(ms / t_all, 4), "achieved_gbs": None if ach is None else round(ach, 1),
+                         "frac": None if ach is None else round(ach / peak, 4)}
+    dom_name = next(iter(kernels))
+    dom_ms, dom_n = per_kernel[dom_name]
+    dom_bytes = kernel_alg_bytes(dom_name, sweep_bytes, msg_by_kind, dense_bytes, emit_read_frac, adaptive_topk)
     dom_avg_s = dom_ms / dom_n * 1e-3
-    achieved = dom_bytes / dom_avg_s / 1e9
-    ratio = NCU_TRAFFIC_RATIO.get(f"{dom_name}:{w.dtype}")
-    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "peak_source": peak_kind,
-                "traffic": None if ratio is None else ratio * dom_bytes,
+    achieved = None if not dom_bytes else dom_bytes / dom_avg_s / 1e9
+    ratio = ratios.get(f"{dom_name}:{w.dtype}")
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": None if achieved is None else round(achieved, 1),
+                "peak": peak, "unit": "GB/s", "frac": None if achieved is None else round(achieved / peak, 4),
+                "peak_source": peak_kind,
+                "traffic": None if (ratio is None or not dom_bytes) else ratio * dom_bytes,
                 "alg_bytes_per_launch": dom_bytes, "avg_launch_ms": round(dom_avg_s * 1e3, 4)}
     b_alg = sum(sweeps_charged(x, emit_read_frac) * sweep_bytes + dense_bytes for x in subs) + 2 * msg_bytes
     step_frac = b_alg / (ms_per_step * 1e-3) / 1e9 / peak
-    kernels = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] / args.steps,
-                   "share": round(v[0] / sum(x[0] for x in per_kernel.values()), 4)}
-               for k, v in sorted(per_kernel.items(), key=lambda kv: -kv[1][0])}
 
     # ---- end to end: inputs start in pinned host memory, the dense mean ends in host memory
     e2e = None
-    if args.e2e_steps > 0:
+    if e2e_steps > 0:
         host_in = torch.empty(r.batches[0].shape, dtype=r.batches[0].dtype, pin_memory=True)
         host_in.copy_(r.batches[0])
         host_out = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
@@ -343,39 +389,80 @@ def run_cuda(args):
         barrier(world)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for i in range(args.e2e_steps):
+        for i in range(e2e_steps):
             e2e_step(i + 1)
         b.record()
         torch.cuda.synchronize()
         barrier(world)
-        e2e_ms = max_over_ranks(a.elapsed_time(b), world, r.dev) / args.e2e_steps
+        e2e_ms = max_over_ranks(a.elapsed_time(b), world, r.dev) / e2e_steps
         e2e = {"value": round(world * len(subs) * sweep_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
                "h2d_bytes_per_step": int(sweep_bytes), "d2h_bytes_per_step": int(dense_bytes),
                "ms_per_step": round(e2e_ms, 3)}
         del host_in, host_out
 
+    words = describe(subs) + f", L={r.L}"
+    if len(subs) > 1:
+        words += f"; value counts the gradient bytes once per variant ({len(subs)} x M*d*4 per step)"
+    res = {
+        "value": round(value, 2), "ms_per_step": round(ms_per_step, 4), "steps": steps,
+        "config": {"workload": words, "l2_policy": l2_policy(sweep_bytes, len(r.batches)),
+                   "parallelism": "replicas only"},
+        "elements_per_s": round(world * len(subs) * w.M * w.d / (ms_per_step * 1e-3), 1),
+        "step_roofline": {"alg_bytes_per_step": b_alg,
+                          "sweeps_charged": [round(sweeps_charged(x, emit_read_frac), 3) for x in subs],
+                          "emit_tiles_read_frac": None if emit_read_frac is None else round(emit_read_frac, 4),
+                          "message_bytes_per_step": msg_bytes, "frac_of_peak": round(step_frac, 4),
+                          "frac_of_8TBs": round(b_alg / (ms_per_step * 1e-3) / 8e12, 4)},
+        "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "e2e": e2e, "clocks": clocks,
+        "device_status": status, "wall_s_timed": round(t_wall, 3),
+    }
+    row0 = r.batches[0][0].clone() if (rank == 0 and world == 1) else None
+    r.close()
+    del r, flush
+    torch.cuda.empty_cache()
+    return res, row0
+
+
+def run_cuda(args):
+    import torch
+    from paper_2507_05508_b200 import build as cuda_build
+    from paper_2507_05508_b200 import workloads as wl
+    cuda_build.build()
+    rank, world, local = dist_setup(args.gpus)
+    subs = sub_workloads(args.workload)
+    if args.shrink_d or args.shrink_M:
+        subs = [wl.shrink(x, args.shrink_d or x.d, args.shrink_M or x.M) for x in subs]
+    w = subs[0]
+    peak, peak_kind = measured_peak()
+    res, row0 = measure(subs, local, rank, world, args.steps, args.warmup, peak, peak_kind, args.e2e_steps)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(subs, r.batches[0][0], budget_s=15.0)
+        cpu = cpu_baseline(subs, row0, budget_s=15.0)
+    del row0
+
+    # the other benchmark workloads, shorter runs of the same measurement (single GPU, default workload only)
+    also = None
+    if world == 1 and args.workload == "c5" and not args.no_also and not (args.shrink_d or args.shrink_M):
+        also = {}
+        for name in ("c4", "c5a", "c5b", "c3"):
+            r2, _ = measure(sub_workloads(name), local, rank, world, args.also_steps, 3, peak, peak_kind, 0)
+            also[name] = {k: r2[k] for k in ("ms_per_step", "value", "steps", "config", "step_roofline", "roofline",
+                                            "gpu_launches", "device_status")}
+            also[name]["kernels"] = {k: v for k, v in list(r2["kernels"].items())[:6]}
+            also[name]["clocks"] = {k: r2["clocks"].get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons")}
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+            "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16",
-            "data": "synthetic",
-            "config": {"workload": describe(subs) + f", L={r.L}", "l2_policy": "inputs larger than L2: "
-                       f"{sweep_bytes / 1e6:.0f} MB per sweep, 2 batches alternated", "parallelism": "replicas only"},
-            "elements_per_s": round(world * len(subs) * w.M * w.d / (ms_per_step * 1e-3), 1),
-            "step_roofline": {"alg_bytes_per_step": b_alg, "sweeps_charged": [round(sweeps_charged(x, emit_read_frac), 3) for x in subs],
-                              "emit_tiles_read_frac": None if emit_read_frac is None else round(emit_read_frac, 4),
-                              "message_bytes_per_step": msg_bytes, "frac_of_peak": round(step_frac, 4),
-                              "frac_of_8TBs": round(b_alg / (ms_per_step * 1e-3) / 8e12, 4)},
-            "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "e2e": e2e,
-            "cpu_baseline": cpu, "clocks": clocks, "device_status": status, "wall_s_timed": round(t_wall, 3),
+            "data": "synthetic", "config": res["config"], "elements_per_s": res["elements_per_s"],
+            "step_roofline": res["step_roofline"], "roofline": res["roofline"], "kernels": res["kernels"],
+            "gpu_launches": res["gpu_launches"], "e2e": res["e2e"], "cpu_baseline": cpu, "clocks": res["clocks"],
+            "device_status": res["device_status"], "wall_s_timed": res["wall_s_timed"], "also": also,
         }
         print(json.dumps(line))
-    r.close()
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
