@@ -88,8 +88,15 @@ __device__ __forceinline__ void load_batch(const T* __restrict__ row, int64_t d,
     }
 }
 
-// Starts the copy of batch `batch` of tile `tile` into a warp's shared-memory slot (kBatchWords words, word i at
-// slot[i]): 16-byte asynchronous copies, or plain padded stores for the ragged end of the row.
+// The write pass gives every lane 16 consecutive words of a batch (four 16-byte chunks), so that the order of the
+// lanes is the order of the coordinates.  Chunk c = 4 * lane + j of the batch is kept at position swz(c) of the
+// warp's shared-memory slot: with the two low bits of the chunk number XOR-ed with bits 3..4, the eight lanes of a
+// quarter warp read their j-th chunks (128-bit loads, 64 bytes apart before the swizzle) from eight different
+// 16-byte bank groups.
+__device__ __forceinline__ int swz(int c) { return (c & ~3) | ((c ^ (c >> 3)) & 3); }
+
+// Starts the copy of batch `batch` of tile `tile` into a warp's shared-memory slot (kBatchWords words in the
+// swizzled chunk order above): 16-byte asynchronous copies, or plain padded stores for the ragged end of the row.
 template <typename T>
 __device__ __forceinline__ void copy_batch_async(const T* __restrict__ row, int64_t d, int64_t tile, int batch, int lane,
                                                  uint32_t* slot) {
@@ -98,7 +105,7 @@ __device__ __forceinline__ void copy_batch_async(const T* __restrict__ row, int6
     const uint32_t* words = reinterpret_cast<const uint32_t*>(row) + w0;
     if ((w0 + kBatchWords) * EW::S <= d) {
 #pragma unroll
-        for (int c = lane; c < kBatchWords / 4; c += 32) cp_async_16(slot + c * 4, words + c * 4);
+        for (int c = lane; c < kBatchWords / 4; c += 32) cp_async_16(slot + swz(c) * 4, words + c * 4);
     } else {
         for (int i = lane; i < kBatchWords; i += 32) {
             const int64_t wi = w0 + i;
@@ -108,7 +115,7 @@ __device__ __forceinline__ void copy_batch_async(const T* __restrict__ row, int6
             } else if (EW::S == 2 && wi * 2 < d) {  // odd bf16 tail: only the low half exists
                 v = (uint32_t)reinterpret_cast<const uint16_t*>(row)[wi * 2] | 0x7FFF0000u;
             }
-            slot[i] = v;
+            slot[swz(i >> 2) * 4 + (i & 3)] = v;
         }
     }
 }
@@ -161,6 +168,50 @@ __device__ __forceinline__ uint32_t batch_flags(const uint32_t (&w)[kEmitRows], 
     }
     *cA = a;
     *cB = b;
+    return flags;
+}
+
+// The same flags for the write pass, with the ties as masks instead of counts: bit i (fp32) or bits i and 16 + i
+// (bf16 low / high half) of mA / mB = word i of this lane holds a key equal to Ta / Tb.
+template <typename T>
+__device__ __forceinline__ uint32_t batch_masks(const uint32_t (&w)[kEmitRows], uint32_t Tb, uint32_t Ta, uint32_t* mA,
+                                                uint32_t* mB) {
+    uint32_t flags = 0, a = 0, b = 0;
+    if constexpr (EmitWord<T>::S == 1) {
+        const uint32_t W = Ta - Tb;
+#pragma unroll
+        for (int i = 0; i < kEmitRows; ++i)
+            if (((w[i] & 0x7FFFFFFFu) - Tb) <= W) flags |= 1u << i;
+        if (__any_sync(0xFFFFFFFFu, flags != 0u)) {
+#pragma unroll
+            for (int i = 0; i < kEmitRows; ++i) {
+                const uint32_t tk = (w[i] & 0x7FFFFFFFu) - Tb;
+                a |= (tk == W) ? (1u << i) : 0u;
+                b |= (tk == 0u) ? (1u << i) : 0u;
+            }
+        }
+    } else {
+        const uint32_t hi = 0x80008000u;
+        const uint32_t geB = hi - Tb * 0x10001u, geB1 = hi - (Tb + 1u) * 0x10001u;
+        const uint32_t leA = hi + Ta * 0x10001u, leA1 = hi + (Ta ? Ta - 1u : 0u) * 0x10001u;
+        const uint32_t keepA1 = Ta ? 0xFFFFFFFFu : 0u;  // Ta = 0: every closed key equals Ta
+#pragma unroll
+        for (int i = 0; i < kEmitRows; ++i) {
+            const uint32_t k2 = w[i] & 0x7FFF7FFFu;
+            flags |= ((k2 + geB) & (leA - k2) & hi) >> (15 - i);
+        }
+        if (__any_sync(0xFFFFFFFFu, flags != 0u)) {
+#pragma unroll
+            for (int i = 0; i < kEmitRows; ++i) {
+                const uint32_t k2 = w[i] & 0x7FFF7FFFu;
+                const uint32_t f = (k2 + geB) & (leA - k2) & hi;
+                b |= (f & ~(k2 + geB1)) >> (15 - i);
+                a |= (f & ~((leA1 - k2) & keepA1)) >> (15 - i);
+            }
+        }
+    }
+    *mA = a;
+    *mB = b;
     return flags;
 }
 
@@ -329,8 +380,10 @@ band_scan_kernel(uint4* __restrict__ rec, int tiles_per_worker, const uint32_t* 
     }
 }
 
-// Pass 3: every listed tile is read again and its band entries are written at their final positions.  Within a
-// row of 32 words the entries are consecutive, so the stores coalesce.
+// Pass 3: every listed tile is read again and its band entries are written at their final positions.
+// A lane owns 16 consecutive words of a batch, so the order of the lanes is the order of the coordinates: the
+// position of a lane's first entry is the batch's base plus the entries of the lanes before it (one warp scan per
+// batch), and the lane then writes its own entries one after the other.
 template <typename T>
 __global__ void __launch_bounds__(kBandThreads)
 band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker,
@@ -339,15 +392,17 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
                   uint32_t* __restrict__ idx_out, float* __restrict__ val_out, int64_t capacity) {
     using EW = EmitWord<T>;
     constexpr int S = EW::S;
+    static_assert(kEmitRows == 16, "a lane owns four 16-byte chunks of a batch");
     // every warp stages its batches in a ring of three shared-memory slots: two copies are in flight while a
-    // batch is ranked, and the rows of a batch can be addressed by a run-time index
+    // batch is ranked, and the words of a batch can be addressed by a run-time index
     extern __shared__ __align__(16) uint32_t sh_dyn[];  // [warps][3][kBatchWords] ring, then sh_off[M + 1]
     uint32_t* sh_off = sh_dyn + (kBandThreads / 32) * kWriteSlots * kBatchWords;
     list_offsets(tile_n, M, sh_off);
     const uint32_t total = sh_off[M];
     const int lane = threadIdx.x & 31;
     uint32_t* ring = sh_dyn + (threadIdx.x >> 5) * kWriteSlots * kBatchWords;
-    const uint32_t lt = (1u << lane) - 1u;
+    // where this lane's words sit in a slot: word r at own + (r ^ own_xor), i.e. chunk q at swz(4 * lane + q)
+    const int own = lane * kEmitRows, own_xor = ((lane >> 1) & 3) << 2;
     const uint32_t warps = gridDim.x * (kBandThreads / 32);
     for (uint32_t f = blockIdx.x * (kBandThreads / 32) + (threadIdx.x >> 5); f < total; f += warps) {
         const int m = worker_of(sh_off, M, f);
@@ -374,146 +429,88 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
             cp_async_commit();  // one group per step, empty at the end of the tile
             cp_async_wait<2>();  // batch b has landed
             __syncwarp();
-            const uint32_t* slot = ring + (b % kWriteSlots) * kBatchWords + lane;
+            const uint32_t* slot = ring + (b % kWriteSlots) * kBatchWords;
             uint32_t cur[kEmitRows];
 #pragma unroll
-            for (int r = 0; r < kEmitRows; ++r) cur[r] = slot[r * 32];
-            uint32_t a1, b1;
-            const uint32_t flags = batch_flags<T>(cur, Tb, Ta, &a1, &b1);
-            const uint32_t rowany = __reduce_or_sync(0xFFFFFFFFu, flags);
-            if (rowany) {  // warp-uniform
-                const uint32_t totCA = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(flags) | (a1 << 16));
-                const uint32_t myB = __reduce_add_sync(0xFFFFFFFFu, b1);
-                const uint32_t myC = totCA & 0xFFFFu, myA = totCA >> 16;
-                uint32_t base = band_prefix(rC, rA, rB, ep.ra, ep.rb);
+            for (int q = 0; q < 4; ++q) {
+                const uint4 x = *reinterpret_cast<const uint4*>(slot + own + ((4 * q) ^ own_xor));
+                cur[4 * q + 0] = x.x; cur[4 * q + 1] = x.y; cur[4 * q + 2] = x.z; cur[4 * q + 3] = x.w;
+            }
+            uint32_t mA, mB;
+            uint32_t member = batch_masks<T>(cur, Tb, Ta, &mA, &mB);
+            if (!__any_sync(0xFFFFFFFFu, member != 0u)) continue;  // no closed-range key in the batch: nothing to count either
+            const uint32_t nC = __popc(member), nA = __popc(mA), nB = __popc(mB);
+            const uint32_t totCA = __reduce_add_sync(0xFFFFFFFFu, nC | (nA << 16));
+            const uint32_t myB = __reduce_add_sync(0xFFFFFFFFu, nB);
+            const uint32_t myC = totCA & 0xFFFFu, myA = totCA >> 16;
+            const uint32_t base = band_prefix(rC, rA, rB, ep.ra, ep.rb);
+            if ((myA | myB) != 0u) {  // warp-uniform
                 // Ties in this batch.  Unless the cut rank of a threshold falls among them, all of them are on one
                 // side of it: the ties of Ta all outside Top-k_{l-1} (in the band) or all inside (dropped), the ties
                 // of Tb all inside Top-k_l (in the band) or all outside (dropped).  Only a batch that holds a cut
                 // ranks its ties one by one.
                 const bool dropA = myA != 0u && rA + myA <= ep.ra, keepA = myA == 0u || rA >= ep.ra;
                 const bool dropB = myB != 0u && rB >= ep.rb, keepB = myB == 0u || rB + myB <= ep.rb;
-                const bool ties = !((keepA || dropA) && (keepB || dropB)) || ((myA | myB) != 0u && W == 0u);
-                const bool drop_any = !ties && (dropA || dropB);
-                uint32_t tA = rA, tB = rB;  // tie ranks, advanced row by row on the ties path
-                const uint32_t e0 = (uint32_t)((tile * kEmitTile + (int64_t)b * kBatchWords + lane) * S);
-                uint32_t rows = (rowany | (rowany >> 16)) & 0xFFFFu;  // rows that hold a closed-range key
-                if (!ties) {
-                    // No tie needs ranking: membership follows from the entry's own key.  Two rows per trip, so that
-                    // the ballots and counts of one row do not wait for the position arithmetic of the other.
-                    auto member = [&](uint32_t w, int i, int s) -> bool {
-                        bool em = (flags >> (i + 16 * s)) & 1u;
-                        if (drop_any) {  // warp-uniform
-                            const uint32_t tk = EW::key(w, s) - Tb;
-                            em = em && !(dropA && tk == W) && !(dropB && tk == 0u);
-                        }
-                        return em;
-                    };
-#pragma unroll 1
+                const bool ranked = !((keepA || dropA) && (keepB || dropB)) || W == 0u;
+                if (!ranked) {
+                    if (dropA) member &= ~mA;
+                    if (dropB) member &= ~mB;
+                } else {
+                    // index-ordered tie ranks (0-based): the ties of the lanes before this one, then this lane's in order
+                    uint32_t iA = nA, iB = nB;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t yA = __shfl_up_sync(0xFFFFFFFFu, iA, o), yB = __shfl_up_sync(0xFFFFFFFFu, iB, o);
+                        if (lane >= o) { iA += yA; iB += yB; }
+                    }
+                    uint32_t tA = rA + iA - nA, tB = rB + iB - nB;
+                    const uint32_t t = mA | mB;
+                    uint32_t rows = (S == 1) ? t : ((t | (t >> 16)) & 0xFFFFu);
                     while (rows) {
-                        constexpr int R = 2;  // rows per trip (four need 74 registers and lose a resident block)
-                        int ri[R];
-                        bool on[R];  // warp-uniform
-                        uint32_t wv[R];
+                        const int r = __ffs(rows) - 1;
+                        rows &= rows - 1u;
 #pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            on[r] = rows != 0u;
-                            ri[r] = on[r] ? __ffs(rows) - 1 : 0;
-                            if (on[r]) rows &= rows - 1u;
-                            wv[r] = slot[ri[r] * 32];
-                        }
-                        bool em[R][S];
-                        uint32_t below[R], cnt[R];
-#pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            below[r] = 0;
-                            cnt[r] = 0;
-#pragma unroll
-                            for (int s = 0; s < S; ++s) {
-                                em[r][s] = on[r] && member(wv[r], ri[r], s);
-                                const uint32_t mk = __ballot_sync(0xFFFFFFFFu, em[r][s]);
-                                below[r] += __popc(mk & lt);
-                                cnt[r] += __popc(mk);
+                        for (int s = 0; s < S; ++s) {
+                            const uint32_t bit = 1u << (r + 16 * s);
+                            if (mA & bit) {
+                                if (tA < ep.ra) member &= ~bit;   // still inside Top-k_{l-1}
+                                ++tA;
                             }
-                        }
-#pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            uint32_t pos = base + below[r];
-                            base += cnt[r];  // the base of the next row
-#pragma unroll
-                            for (int s = 0; s < S; ++s) {
-                                if (em[r][s]) {
-                                    if ((int64_t)pos < capacity) {
-                                        idx_w[pos] = e0 + (uint32_t)(ri[r] * 32 * S + s);
-                                        val_w[pos] = EW::value(wv[r], s) * inv_p;
-                                    }
-                                    ++pos;
-                                }
+                            if (mB & bit) {
+                                if (tB >= ep.rb) member &= ~bit;  // already outside Top-k_l
+                                ++tB;
                             }
                         }
                     }
                 }
-                // ties to rank: a rolled loop over the rows that matter, each row continuing from the one before
-                // (the body is long, unrolling it 16 times would not fit the instruction cache)
-#pragma unroll 1
-                while (rows) {
-                    const int i = __ffs(rows) - 1;
-                    rows &= rows - 1u;
-                    const uint32_t w = slot[i * 32];
-                    bool em[S];
-                    uint32_t me[S];
-                    if (!ties) {
-#pragma unroll
-                        for (int s = 0; s < S; ++s) {
-                            em[s] = (flags >> (i + 16 * s)) & 1u;
-                            if (drop_any) {  // warp-uniform
-                                const uint32_t tk = EW::key(w, s) - Tb;
-                                em[s] = em[s] && !(dropA && tk == W) && !(dropB && tk == 0u);
-                            }
-                            me[s] = __ballot_sync(0xFFFFFFFFu, em[s]);
-                        }
-                    } else {
-                        uint32_t tk[S], mA[S], mB[S], a_lt = 0, b_lt = 0;
-#pragma unroll
-                        for (int s = 0; s < S; ++s) {
-                            tk[s] = EW::key(w, s) - Tb;
-                            mA[s] = __ballot_sync(0xFFFFFFFFu, tk[s] == W);
-                            mB[s] = __ballot_sync(0xFFFFFFFFu, tk[s] == 0u);
-                            a_lt += __popc(mA[s] & lt);
-                            b_lt += __popc(mB[s] & lt);
-                        }
-#pragma unroll
-                        for (int s = 0; s < S; ++s) {
-                            // index-ordered tie ranks (0-based) of this element among the keys equal to Ta / Tb
-                            const bool inA = (tk[s] == W) && (tA + a_lt) < ep.ra;    // still inside Top-k_{l-1}
-                            const bool outB = (tk[s] == 0u) && (tB + b_lt) >= ep.rb; // already outside Top-k_l
-                            em[s] = (tk[s] <= W) && !inA && !outB;
-                            me[s] = __ballot_sync(0xFFFFFFFFu, em[s]);
-                            a_lt += (mA[s] >> lane) & 1u;
-                            b_lt += (mB[s] >> lane) & 1u;
-                        }
-#pragma unroll
-                        for (int s = 0; s < S; ++s) {
-                            tA += __popc(mA[s]);
-                            tB += __popc(mB[s]);
-                        }
-                    }
-                    uint32_t pos = base;
-#pragma unroll
-                    for (int s = 0; s < S; ++s) pos += __popc(me[s] & lt);
-#pragma unroll
-                    for (int s = 0; s < S; ++s) {
-                        if (em[s]) {
-                            if ((int64_t)pos < capacity) {
-                                idx_w[pos] = e0 + (uint32_t)(i * 32 * S + s);
-                                val_w[pos] = EW::value(w, s) * inv_p;
-                            }
-                            ++pos;
-                        }
-                    }
-                    base = __shfl_sync(0xFFFFFFFFu, pos, 31);  // lane 31 ends at the row's total
-                }
-                rC += myC; rA += myA; rB += myB;
             }
+            // positions: the batch's base plus the entries of the lanes before this one
+            const uint32_t cnt = __popc(member);
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += y;
+            }
+            uint32_t pos = base + incl - cnt;
+            const uint32_t e0 = (uint32_t)((tile * kEmitTile + (int64_t)b * kBatchWords + lane * kEmitRows) * S);
+            uint32_t rows = (S == 1) ? member : ((member | (member >> 16)) & 0xFFFFu);
+            while (rows) {  // this lane's words that hold an entry, in ascending order
+                const int r = __ffs(rows) - 1;
+                rows &= rows - 1u;
+                const uint32_t w = slot[own + (r ^ own_xor)];  // word r of this lane in the swizzled slot
+#pragma unroll
+                for (int s = 0; s < S; ++s) {
+                    if ((member >> (r + 16 * s)) & 1u) {
+                        if ((int64_t)pos < capacity) {
+                            idx_w[pos] = e0 + (uint32_t)(r * S + s);
+                            val_w[pos] = EW::value(w, s) * inv_p;
+                        }
+                        ++pos;
+                    }
+                }
+            }
+            rC += myC; rA += myA; rB += myB;
         }
     }
     cp_async_wait<0>();
@@ -574,6 +571,76 @@ aggregate_topk_kernel(const uint32_t* __restrict__ idx, const float* __restrict_
                 if (base + i < d) out[base + i] = acc[i] * inv_M;
         }
         __syncthreads();
+    }
+}
+
+
+// The same average without a block barrier per worker: every warp owns kAggSub consecutive coordinates of the
+// tile and adds the workers' entries that fall into them in worker order 0..M-1 (the order of the fp32 additions per
+// coordinate is the same as in the kernel above, so the two give identical results).  Lane l finds, for worker
+// m0 + l, where the warp's coordinates begin and end inside that worker's slice of the tile (two binary searches in
+// an index-sorted slice); the warp then walks the workers one after the other.
+constexpr int kAggSub = 512;
+constexpr int kAggWarps = kAggTile / kAggSub;
+
+__global__ void __launch_bounds__(kAggWarps * 32)
+aggregate_topk_warps_kernel(const uint32_t* __restrict__ idx, const float* __restrict__ val, int64_t capacity, int M,
+                            int64_t d, int ntiles, const uint32_t* __restrict__ offsets, float* __restrict__ out) {
+    __shared__ __align__(16) float acc_all[kAggTile];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* acc = acc_all + warp * kAggSub;
+    const float inv_M = 1.0f / (float)M;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const int64_t base = (int64_t)t * kAggTile + (int64_t)warp * kAggSub;  // first coordinate of this warp
+#pragma unroll
+        for (int i = 0; i < kAggSub / 128; ++i)
+            reinterpret_cast<float4*>(acc)[i * 32 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncwarp();
+        if (base < d) {
+            for (int m0 = 0; m0 < M; m0 += 32) {
+                const int m = m0 + lane;
+                uint32_t s0 = 0, s1 = 0;
+                if (m < M) {
+                    const uint32_t o0 = offsets[(int64_t)m * (ntiles + 1) + t], o1 = offsets[(int64_t)m * (ntiles + 1) + t + 1];
+                    const uint32_t* a = idx + (int64_t)m * capacity;
+                    auto first_at_least = [&](uint64_t target) -> uint32_t {
+                        uint32_t lo = o0, hi = o1;
+                        while (lo < hi) {
+                            const uint32_t mid = lo + ((hi - lo) >> 1);
+                            if ((uint64_t)__ldg(&a[mid]) < target) lo = mid + 1; else hi = mid;
+                        }
+                        return lo;
+                    };
+                    s0 = (warp == 0) ? o0 : first_at_least((uint64_t)base);
+                    s1 = (warp == kAggWarps - 1) ? o1 : first_at_least((uint64_t)base + kAggSub);
+                }
+                const int nm = min(32, M - m0);
+                for (int mm = 0; mm < nm; ++mm) {  // fixed worker order: reproducible fp32 sums
+                    const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, s0, mm), b1 = __shfl_sync(0xFFFFFFFFu, s1, mm);
+                    if (b1 > b0) {  // warp-uniform
+                        const uint32_t* a = idx + (int64_t)(m0 + mm) * capacity;
+                        const float* v = val + (int64_t)(m0 + mm) * capacity;
+                        for (uint32_t j = b0 + lane; j < b1; j += 32) {
+                            const uint32_t off = __ldg(&a[j]) - (uint32_t)base;  // indices are unique within a worker
+                            if (off < (uint32_t)kAggSub) acc[off] += __ldg(&v[j]);  // an unsorted message cannot reach outside
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+        }
+        if (base + kAggSub <= d && (d & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < kAggSub / 128; ++i) {
+                float4 x = reinterpret_cast<const float4*>(acc)[i * 32 + lane];
+                x.x *= inv_M; x.y *= inv_M; x.z *= inv_M; x.w *= inv_M;
+                reinterpret_cast<float4*>(out + base)[i * 32 + lane] = x;
+            }
+        } else {
+            for (int i = lane; i < kAggSub; i += 32)
+                if (base + i < d) out[base + i] = acc[i] * inv_M;
+        }
+        __syncwarp();
     }
 }
 
@@ -648,8 +715,8 @@ void launch_aggregate_topk(Workspace& ws, const mlmc_topk_msgs& msgs, int M, int
     int grid = ws.sm_count * 8;
     if (grid > ntiles) grid = ntiles;
     LaunchScope t(ws, K_AGG_TOPK, s);
-    aggregate_topk_kernel<<<grid, 256, 2 * M * sizeof(uint32_t), s>>>(msgs.idx, msgs.val, msgs.capacity, M, d, ntiles,
-                                                                      ws.agg_offsets, out);
+    aggregate_topk_warps_kernel<<<grid, kAggWarps * 32, 0, s>>>(msgs.idx, msgs.val, msgs.capacity, M, d, ntiles,
+                                                                ws.agg_offsets, out);
 }
 
 }  // namespace mlmc
