@@ -204,3 +204,128 @@ def aggregate_bitwise(msgs, b, d):
     _check(lib().mlmc_oracle_aggregate_bitwise(C.c_int(M), pp, _ptr(gmax), _ptr(level), _ptr(p_sel), _ptr(b),
                                                C.c_int(len(b)), C.c_int64(d), _ptr(out), _ptr(scale)))
     return out, scale
+
+
+# ----------------------------------------------------------------------------------------------
+# floating-point bit-wise MLMC (App. B), s-Top-k (App. D), MLMC-RTN (App. G)
+# ----------------------------------------------------------------------------------------------
+def float_compress(g, keep: int):
+    """Dense C(g) that keeps sign, exponent and the first `keep` mantissa digits (fp64 copy)."""
+    g, dt = _as_input(g)
+    out = np.empty(g.size)
+    _check(lib().mlmc_oracle_float_compress(_ptr(g), C.c_int(dt), C.c_int64(g.size), C.c_int(keep), _ptr(out)))
+    return out
+
+
+@dataclass
+class FloatMsg:
+    level: int
+    p_sel: float
+    u: float
+    margin: float
+    p: np.ndarray
+    expo: np.ndarray     # uint8[d]
+    planes: np.ndarray   # [1 + w_level][ceil(d/32)] uint32
+    est: np.ndarray      # fp64[d]: g^0 + (C^l - C^{l-1}) / p_l
+
+
+def floatbits(g, mb, p=None, seed=0, step=0, worker=0, force_level=-1) -> FloatMsg:
+    g, dt = _as_input(g)
+    d = g.size
+    mb = np.ascontiguousarray(mb, dtype=np.int32)
+    L = len(mb)
+    p_in = None if p is None else np.ascontiguousarray(p, dtype=np.float64)
+    widths = np.diff(np.concatenate([[0], mb]))
+    w_max = int(widths.max())
+    words = (d + 31) // 32
+    planes = np.zeros((1 + w_max, words), dtype=np.uint32)
+    expo = np.empty(d, dtype=np.uint8)
+    est = np.empty(d)
+    p_out = np.empty(L)
+    level = C.c_int32()
+    p_sel, u, margin = C.c_double(), C.c_double(), C.c_double()
+    _check(lib().mlmc_oracle_floatbits(
+        _ptr(g), C.c_int(dt), C.c_int64(d), _ptr(mb), C.c_int(L), _ptr(p_in),
+        C.c_uint64(seed), C.c_uint64(step), C.c_uint64(worker), C.c_int(force_level),
+        _ptr(p_out), C.byref(level), C.byref(p_sel), C.byref(u), C.byref(margin),
+        _ptr(expo), _ptr(planes), C.c_int32(w_max), _ptr(est)))
+    w = int(widths[level.value])
+    return FloatMsg(level.value, p_sel.value, u.value, margin.value, p_out, expo, planes[:1 + w].copy(), est)
+
+
+def floatbits_decode(expo, planes, d, mb, level, p_sel, bf16=False):
+    expo = np.ascontiguousarray(expo, dtype=np.uint8)
+    planes = np.ascontiguousarray(planes, dtype=np.uint32)
+    mb = np.ascontiguousarray(mb, dtype=np.int32)
+    est = np.empty(d)
+    _check(lib().mlmc_oracle_floatbits_decode(_ptr(expo), _ptr(planes), C.c_int64(d), C.c_int(BF16 if bf16 else F32),
+                                              _ptr(mb), C.c_int(len(mb)), C.c_int(level), C.c_double(p_sel), _ptr(est)))
+    return est
+
+
+def aggregate_dense(rows, d):
+    """rows: list of fp64[d] (or fp32) dense estimates.  Returns (mean fp64[d], scale fp64[d])."""
+    rows = [np.ascontiguousarray(r, dtype=np.float64) for r in rows]
+    M = len(rows)
+    rp = (C.c_void_p * M)(*[r.ctypes.data for r in rows])
+    out, scale = np.empty(d), np.empty(d)
+    _check(lib().mlmc_oracle_aggregate_dense(C.c_int(M), rp, C.c_int64(d), _ptr(out), _ptr(scale)))
+    return out, scale
+
+
+def stopk(g, s: int, p=None, seed=0, step=0, worker=0, force_level=-1) -> TopkMsg:
+    g, dt = _as_input(g)
+    d = g.size
+    L = (d + s - 1) // s
+    p_in = None if p is None else np.ascontiguousarray(p, dtype=np.float64)
+    p_out, delta = np.empty(L), np.empty(L)
+    level, count = C.c_int32(), C.c_int64()
+    p_sel, u, margin = C.c_double(), C.c_double(), C.c_double()
+    idx = np.empty(s, dtype=np.uint32)
+    val = np.empty(s, dtype=np.float32)
+    _check(lib().mlmc_oracle_stopk(
+        _ptr(g), C.c_int(dt), C.c_int64(d), C.c_int64(s), _ptr(p_in),
+        C.c_uint64(seed), C.c_uint64(step), C.c_uint64(worker), C.c_int(force_level),
+        _ptr(p_out), _ptr(delta), C.byref(level), C.byref(p_sel), C.byref(u), C.byref(margin),
+        C.byref(count), _ptr(idx), _ptr(val), C.c_int64(s)))
+    n = count.value
+    return TopkMsg(level.value, p_sel.value, u.value, margin.value, p_out, delta, idx[:n].copy(), val[:n].copy())
+
+
+def rtn_compress(g, r, level: int):
+    """Dense C^level(g) for the RTN widths r (len L-1; level L-1 is the identity), fp64."""
+    g, dt = _as_input(g)
+    r = np.ascontiguousarray(r, dtype=np.int32)
+    out = np.empty(g.size)
+    _check(lib().mlmc_oracle_rtn_compress(_ptr(g), C.c_int(dt), C.c_int64(g.size), _ptr(r), C.c_int(len(r) + 1),
+                                          C.c_int(level), _ptr(out)))
+    return out
+
+
+@dataclass
+class RtnMsg:
+    level: int
+    p_sel: float
+    u: float
+    margin: float
+    p: np.ndarray
+    delta: np.ndarray
+    c: float
+    val: np.ndarray      # float32[d]: (C^l - C^{l-1}) / p_l
+
+
+def rtn(g, r, p=None, seed=0, step=0, worker=0, force_level=-1) -> RtnMsg:
+    g, dt = _as_input(g)
+    d = g.size
+    r = np.ascontiguousarray(r, dtype=np.int32)
+    L = len(r) + 1
+    p_in = None if p is None else np.ascontiguousarray(p, dtype=np.float64)
+    p_out, delta = np.empty(L), np.empty(L)
+    val = np.empty(d, dtype=np.float32)
+    level, c = C.c_int32(), C.c_float()
+    p_sel, u, margin = C.c_double(), C.c_double(), C.c_double()
+    _check(lib().mlmc_oracle_rtn(
+        _ptr(g), C.c_int(dt), C.c_int64(d), _ptr(r), C.c_int(L), _ptr(p_in),
+        C.c_uint64(seed), C.c_uint64(step), C.c_uint64(worker), C.c_int(force_level),
+        _ptr(p_out), _ptr(delta), C.byref(level), C.byref(p_sel), C.byref(u), C.byref(margin), C.byref(c), _ptr(val)))
+    return RtnMsg(level.value, p_sel.value, u.value, margin.value, p_out, delta, c.value, val)

@@ -681,41 +681,48 @@ norm_sweep_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const Quer
 }
 
 // bf16: every key is a histogram bin, so the open-interval sums follow from the counts exactly.
-// Per interval every warp adds up its 32 threads' shares by shuffles; after one barrier thread l adds the 32 warp
-// sums of interval l in warp order (a fixed order: reproducible).
-__global__ void __launch_bounds__(kResolveThreads, 1)
+// kNormParts blocks per worker, each over a contiguous 1 / kNormParts of the bins; a bin lies in exactly one open
+// interval (or is a threshold), found by a search over the thresholds.  Per interval every warp adds up its lanes'
+// shares by shuffles; after one barrier thread l adds the warp sums of interval l in warp order, and the draw
+// kernel adds the kNormParts partials in block order (fixed orders: reproducible).
+constexpr int kNormParts = 8;
+constexpr int kNormThreads = 256;
+
+__global__ void __launch_bounds__(kNormThreads)
 norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query* queries, int L,
                            double* band_partial, int norm_ctas, const int* worker_err) {
-    __shared__ double sh_part[kMaxLevels][kResolveThreads / 32];
+    __shared__ double sh_part[kMaxLevels][kNormThreads / 32];
     __shared__ uint32_t sh_thr[kMaxQueries];
-    const int m = blockIdx.x;
+    const int m = blockIdx.y, part = blockIdx.x;
     if (worker_err[m]) return;
     const uint32_t* S = hist1 + (int64_t)m * kBins1;
     if (threadIdx.x < kMaxQueries)
         sh_thr[threadIdx.x] = (threadIdx.x < L - 1) ? queries[m * kMaxQueries + threadIdx.x].T : 0u;
     __syncthreads();
-    constexpr int per = kBins1 / kResolveThreads;
+    constexpr int per = kBins1 / kNormParts / kNormThreads;  // 16 bins per thread, coalesced over the block
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // this thread's keys (coalesced over the block) with their counts and squares, once
-    uint32_t cnt[per];
+    const int nthr = L - 1;
+    double e[per];   // energy of this thread's bins
+    int iv[per];     // their open interval, or -1 (empty bin, threshold bin: added from the counts by the draw kernel)
 #pragma unroll
     for (int i = 0; i < per; ++i) {
-        const uint32_t key = i * kResolveThreads + threadIdx.x;
-        cnt[i] = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
+        const uint32_t key = (uint32_t)part * (kBins1 / kNormParts) + i * kNormThreads + threadIdx.x;
+        const uint32_t cnt = S[key] - ((key == kBins1 - 1) ? 0u : S[key + 1]);
+        int lo = 0, hi = nthr;  // thresholds are descending: first index with T <= key
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (sh_thr[mid] > key) lo = mid + 1; else hi = mid;
+        }
+        const bool is_thr = lo < nthr && sh_thr[lo] == key;
+        iv[i] = (cnt == 0u || is_thr) ? -1 : lo;  // empty bins include the Inf/NaN encodings, whose value must not enter the sum
+        const double x = (double)__uint_as_float(key << 16);
+        e[i] = (double)cnt * (x * x);
     }
     for (int l = 0; l < L; ++l) {
-        // open interval l: T_l < key < T_{l-1}   (T_{-1} = +inf, T_{L-1} = -1: everything below)
-        const uint32_t hi = (l == 0) ? 0xFFFFFFFFu : sh_thr[l - 1];
-        const int64_t lo = (l == L - 1) ? -1 : (int64_t)sh_thr[l];
         double acc = 0.0;
 #pragma unroll
-        for (int i = 0; i < per; ++i) {
-            const uint32_t key = i * kResolveThreads + threadIdx.x;
-            if ((int64_t)key > lo && key < hi && cnt[i]) {  // empty bins include the Inf/NaN encodings, whose value must not enter the sum
-                const double x = (double)__uint_as_float(key << 16);
-                acc = fma((double)cnt[i], x * x, acc);
-            }
-        }
+        for (int i = 0; i < per; ++i)
+            if (iv[i] == l) acc += e[i];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
         if (lane == 0) sh_part[l][warp] = acc;
@@ -723,8 +730,8 @@ norm_from_hist_bf16_kernel(const uint32_t* hist1 /* suffix sums */, const Query*
     __syncthreads();
     if (threadIdx.x < L) {
         double tot = 0.0;
-        for (int w = 0; w < kResolveThreads / 32; ++w) tot += sh_part[threadIdx.x][w];
-        band_partial[((int64_t)m * norm_ctas) * kMaxLevels + threadIdx.x] = tot;
+        for (int w = 0; w < kNormThreads / 32; ++w) tot += sh_part[threadIdx.x][w];
+        band_partial[((int64_t)m * norm_ctas + part) * kMaxLevels + threadIdx.x] = tot;
     }
 }
 
@@ -1051,10 +1058,10 @@ void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int6
 }
 
 void launch_norm_from_hist_bf16(Workspace& ws, int M, int L, cudaStream_t s) {
-    ws.cur_norm_ctas = 1;
+    ws.cur_norm_ctas = kNormParts;
     LaunchScope t(ws, K_NORM_HIST, s);
-    norm_from_hist_bf16_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, L, ws.band_partial, ws.norm_ctas,
-                                                             ws.worker_err);
+    norm_from_hist_bf16_kernel<<<dim3(kNormParts, M), kNormThreads, 0, s>>>(ws.hist1, ws.queries, L, ws.band_partial,
+                                                                            ws.norm_ctas, ws.worker_err);
 }
 
 void launch_probs_draw(Workspace& ws, int dtype, int M, int L, int64_t d, bool adaptive, bool want_emit,
