@@ -40,7 +40,7 @@ extern "C" {
 typedef struct mlmc_ctx mlmc_ctx;
 
 typedef enum { MLMC_F32 = 0, MLMC_BF16 = 1 } mlmc_dtype;
-typedef enum { MLMC_TOPK = 0, MLMC_BITWISE = 1 } mlmc_kind;
+typedef enum { MLMC_TOPK = 0, MLMC_BITWISE = 1, MLMC_RTN = 2 } mlmc_kind;
 
 typedef enum {
     MLMC_OK = 0,
@@ -90,7 +90,8 @@ int mlmc_destroy(mlmc_ctx* ctx);
 int mlmc_get_status(mlmc_ctx* ctx, void* stream);
 
 /* Level probabilities and residual norms (Lemma 3.4; Alg. 3 "Compute p^l = Delta^l / sum Delta").
- *   kind   MLMC_TOPK: sched = host int64 k[L];  MLMC_BITWISE: sched = host int64 b[L].
+ *   kind   MLMC_TOPK: sched = host int64 k[L];  MLMC_BITWISE: sched = host int64 b[L];
+ *          MLMC_RTN: sched = host int64 r[L-1] (the widths of mlmc_compress_rtn; level L-1 is the identity).
  *   p_host NULL: adaptive, p_out[m][l] = Delta_l / sum Delta (all weight on level 0 if every Delta is 0).
  *          else: host double[L], all > 0, sum 1 within 1e-9; p_out[m][l] = p_host[l] / sum.
  *   p_out     device double [M][L].
@@ -123,6 +124,69 @@ int mlmc_compress_bitwise(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, in
  * Workers whose level is -1 contribute nothing. */
 int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, int L, int M, int64_t d,
                    float* out, void* stream);
+
+/* ---- Further multilevel compressors of the paper, same estimator (Eq. 5), same draw, same server average. ---- */
+
+/* s-Top-k (Sec. 2.2 "s-segmented Top-k"; App. D: the segments are those of the sorted vector): level l keeps
+ * the l + 1 segments of length s of largest norm, i.e. Top-(s (l + 1)); L = ceil(d / s) levels; the residual of
+ * level l is the l-th segment (Sec. 3.2), at most s entries, so capacity >= min(s, d) suffices.
+ *   p  host double[L], all > 0, sum 1 (Alg. 2), or NULL for adaptive p (Lemma 3.4: p^l proportional to the norm of
+ *      segment l).  Adaptive p needs every segment norm and is limited to L <= MLMC_MAX_LEVELS; with a given p any
+ *      L up to min(2^20, d_max of the context) is accepted, because the level is drawn before the data is read and
+ *      only the two thresholds of its segment are selected.
+ * Returns MLMC_ERR_ARG when L exceeds those limits. */
+int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int64_t s,
+                        const double* p, uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, void* stream);
+
+/* Floating-point bit-wise message batch (Sec. 2.2 "Floating-point compressors", App. B): sign and exponent of
+ * every entry are always sent, level l adds the mantissa digits mb_{l-1}+1 .. mb_l (one digit per entry for the
+ * unit schedule: the paper's 1 + exponent + 1 bits per entry).
+ *   expo    [M][32 ceil(d/32)] bytes: biased exponent field of entry i of worker m at expo[m * 32 * words + i].
+ *   planes  [M][1 + w_max][ceil(d/32)]: plane 0 = raw sign bits, plane j = bit (w_l - j) of the mantissa field. */
+typedef struct {
+    uint8_t*  expo;
+    uint32_t* planes;
+    int32_t*  level;   /* [M] sampled level, or -1 on a device error (NaN / Inf in g)                 */
+    double*   p_sel;   /* [M]                                                                         */
+    int32_t   w_max;   /* magnitude planes allocated per worker; need >= max_l (mb_l - mb_{l-1})      */
+} mlmc_float_msgs;
+
+/* MLMC with the floating-point compressor (App. B).  C^l(e) keeps sign, exponent and the first mb_l mantissa
+ * digits of every entry; mb host int32[L], strictly increasing, mb[L-1] = 23 for fp32 and 7 for bf16 input (the top
+ * level is the identity, Def. 3.1).  The estimate is g^0 + (1/p^l)(C^l - C^{l-1}) with the always-sent part
+ * g^0 = sign 2^(E - bias) (an entry with exponent field 0 has g^0 = 0 and the scale of exponent field 1).
+ *   p  host double[L] or NULL: NULL takes App. B's optimal fixed probabilities, p^l proportional to 2^-l for the
+ *      unit schedule, in general to the largest residual of the level, 2^-mb_{l-1} - 2^-mb_l.
+ * One sweep over g; the level draw does not depend on the data.  expo and planes must be 16-byte aligned. */
+int mlmc_compress_floatbits(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld,
+                            const int32_t* mb, int L, const double* p, uint64_t seed, uint64_t step,
+                            const mlmc_float_msgs* out, void* stream);
+
+/* Server average of floating-point messages into dense out[d] (fp32, worker order 0..M-1). */
+int mlmc_aggregate_floatbits(mlmc_ctx* ctx, const mlmc_float_msgs* msgs, const int32_t* mb, int L, int M, int64_t d,
+                             float* out, void* stream);
+
+/* MLMC-RTN message batch (Sec. 3.2 end, App. G): the residual of a round-to-nearest level has no sparse or
+ * bit-plane structure, so the message is the dense vector (C^l - C^{l-1}) / p^l. */
+typedef struct {
+    float*   val;      /* [M][ldv] dense residual scaled by 1/p, row stride ldv >= d elements, 16-byte aligned rows */
+    float*   c;        /* [M] clipping value c = max_i |g_i|                                                       */
+    int32_t* level;    /* [M] sampled level, or -1 on a device error                                               */
+    double*  p_sel;    /* [M]                                                                                      */
+    int64_t  ldv;
+} mlmc_rtn_msgs;
+
+/* MLMC with round-to-nearest levels (App. G): C^l(v) = clip(delta^l round(v / delta^l), -c, c),
+ * delta^l = 2c / (2^{r_l} - 1), for bit widths r host int32[L-1], strictly increasing, r <= 16; level L-1 is the
+ * identity (Def. 3.1).  The rounding is fixed as: inv = fl32((2^r - 1) / (2c)), delta = fl32(2c / (2^r - 1)),
+ * t = fl32(v inv), k = t rounded to nearest (ties to even), C = clip(fl32(k delta), -c, c); residuals, their norms
+ * and the scaling by 1/p are fp64, the message value is rounded to fp32 once.
+ *   p  host double[L] or NULL for adaptive p (Lemma 3.4, Alg. 3; the paper's MLMC-RTN is adaptive). */
+int mlmc_compress_rtn(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* r, int L,
+                      const double* p, uint64_t seed, uint64_t step, const mlmc_rtn_msgs* out, void* stream);
+
+/* Server average of dense messages: out[i] = (1/M) sum_m val[m][i], workers with level -1 left out. */
+int mlmc_aggregate_rtn(mlmc_ctx* ctx, const mlmc_rtn_msgs* msgs, int M, int64_t d, float* out, void* stream);
 
 /* The Top-k case of mlmc_aggregate for callers that must not allocate device memory.  (The paper
  * has no counterpart: this is a deployment variant of the same averaging step.)

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmlmc.so")
 
 MLMC_F32, MLMC_BF16 = 0, 1
-MLMC_TOPK, MLMC_BITWISE = 0, 1
+MLMC_TOPK, MLMC_BITWISE, MLMC_RTN = 0, 1, 2
 MLMC_OK = 0
 MLMC_ERR_ARG, MLMC_ERR_SCHEDULE, MLMC_ERR_PROB, MLMC_ERR_CAPACITY = -1, -2, -3, -4
 MLMC_ERR_NONFINITE, MLMC_ERR_TIMEOUT, MLMC_ERR_CUDA, MLMC_ERR_NOMEM, MLMC_ERR_INTERNAL = -5, -6, -7, -8, -9
@@ -25,7 +25,8 @@ MLMC_MAX_LEVELS = 32
 EXPORTS = ["mlmc_create", "mlmc_destroy", "mlmc_get_status", "mlmc_launch_count", "mlmc_read_u", "mlmc_read_listed_tiles",
            "mlmc_kernel_count", "mlmc_kernel_name", "mlmc_timing_enable", "mlmc_timing_read",
            "mlmc_level_probs", "mlmc_compress_topk", "mlmc_compress_bitwise", "mlmc_aggregate",
-           "mlmc_aggregate_topk_noalloc"]
+           "mlmc_aggregate_topk_noalloc", "mlmc_compress_stopk", "mlmc_compress_floatbits", "mlmc_aggregate_floatbits",
+           "mlmc_compress_rtn", "mlmc_aggregate_rtn"]
 
 
 class MlmcError(RuntimeError):
@@ -42,6 +43,16 @@ class mlmc_topk_msgs(C.Structure):
 class mlmc_bit_msgs(C.Structure):
     _fields_ = [("planes", C.c_void_p), ("gmax", C.c_void_p), ("level", C.c_void_p), ("p_sel", C.c_void_p),
                 ("w_max", C.c_int32)]
+
+
+class mlmc_float_msgs(C.Structure):
+    _fields_ = [("expo", C.c_void_p), ("planes", C.c_void_p), ("level", C.c_void_p), ("p_sel", C.c_void_p),
+                ("w_max", C.c_int32)]
+
+
+class mlmc_rtn_msgs(C.Structure):
+    _fields_ = [("val", C.c_void_p), ("c", C.c_void_p), ("level", C.c_void_p), ("p_sel", C.c_void_p),
+                ("ldv", C.c_int64)]
 
 
 _lib = None
@@ -68,6 +79,11 @@ def lib() -> C.CDLL:
         L.mlmc_compress_bitwise.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_aggregate.argtypes = [vp, i32, vp, vp, i32, i32, i64, vp, vp]
         L.mlmc_aggregate_topk_noalloc.argtypes = [vp, i32, i64, vp, vp]
+        L.mlmc_compress_stopk.argtypes = [vp, vp, i32, i64, i32, i64, i64, vp, u64, u64, vp, vp]
+        L.mlmc_compress_floatbits.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
+        L.mlmc_aggregate_floatbits.argtypes = [vp, vp, vp, i32, i32, i64, vp, vp]
+        L.mlmc_compress_rtn.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
+        L.mlmc_aggregate_rtn.argtypes = [vp, vp, i32, i64, vp, vp]
         L.mlmc_kernel_count.argtypes = []
         L.mlmc_kernel_name.argtypes = [i32]
         L.mlmc_timing_enable.argtypes = [vp, i32]
@@ -165,7 +181,8 @@ def mlmc_level_probs(ctx, g: torch.Tensor, kind: int, sched: Sequence[int], p: O
     ptr, dt, d, M, ld = _g_args(g)
     sch = _host_array(C.c_int64, list(sched))
     ph = _host_array(C.c_double, None if p is None else list(p))
-    _check(lib().mlmc_level_probs(ctx, ptr, dt, d, M, ld, kind, sch, len(sched), ph, p_out.data_ptr(),
+    L = len(sched) + (1 if kind == MLMC_RTN else 0)      # the RTN schedule lists the widths below the identity level
+    _check(lib().mlmc_level_probs(ctx, ptr, dt, d, M, ld, kind, sch, L, ph, p_out.data_ptr(),
                                   None if delta_out is None else delta_out.data_ptr(), _stream()), "mlmc_level_probs")
 
 
@@ -199,6 +216,78 @@ def mlmc_aggregate_topk_noalloc(msgs: "TopkBuffers", M: int, d: int, out: torch.
     assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.numel() >= d
     _check(lib().mlmc_aggregate_topk_noalloc(C.byref(msgs.struct), M, d, out.data_ptr(), _stream()),
            "mlmc_aggregate_topk_noalloc")
+
+
+def mlmc_compress_stopk(ctx, g: torch.Tensor, s: int, p: Optional[Sequence[float]], seed: int, step: int,
+                        out: "TopkBuffers") -> None:
+    ptr, dt, d, M, ld = _g_args(g)
+    ph = None if p is None else (C.c_double * len(p)).from_buffer_copy(memoryview(_as_f64(p)))
+    _check(lib().mlmc_compress_stopk(ctx, ptr, dt, d, M, ld, s, ph, seed, step, C.byref(out.struct), _stream()),
+           "mlmc_compress_stopk")
+
+
+def _as_f64(p):
+    import numpy as np
+    return np.ascontiguousarray(p, dtype=np.float64)
+
+
+def mlmc_compress_floatbits(ctx, g: torch.Tensor, mb: Sequence[int], p: Optional[Sequence[float]], seed: int, step: int,
+                            out: "FloatBuffers") -> None:
+    ptr, dt, d, M, ld = _g_args(g)
+    mh = _host_array(C.c_int32, list(mb))
+    ph = _host_array(C.c_double, None if p is None else list(p))
+    _check(lib().mlmc_compress_floatbits(ctx, ptr, dt, d, M, ld, mh, len(mb), ph, seed, step, C.byref(out.struct),
+                                         _stream()), "mlmc_compress_floatbits")
+
+
+def mlmc_aggregate_floatbits(ctx, msgs: "FloatBuffers", mb: Sequence[int], M: int, d: int, out: torch.Tensor) -> None:
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.numel() >= d
+    mh = _host_array(C.c_int32, list(mb))
+    _check(lib().mlmc_aggregate_floatbits(ctx, C.byref(msgs.struct), mh, len(mb), M, d, out.data_ptr(), _stream()),
+           "mlmc_aggregate_floatbits")
+
+
+def mlmc_compress_rtn(ctx, g: torch.Tensor, r: Sequence[int], p: Optional[Sequence[float]], seed: int, step: int,
+                      out: "RtnBuffers") -> None:
+    """r: the L - 1 round-to-nearest widths; level L - 1 is the identity."""
+    ptr, dt, d, M, ld = _g_args(g)
+    rh = _host_array(C.c_int32, list(r)) if len(r) else None
+    ph = _host_array(C.c_double, None if p is None else list(p))
+    _check(lib().mlmc_compress_rtn(ctx, ptr, dt, d, M, ld, rh, len(r) + 1, ph, seed, step, C.byref(out.struct),
+                                   _stream()), "mlmc_compress_rtn")
+
+
+def mlmc_aggregate_rtn(ctx, msgs: "RtnBuffers", M: int, d: int, out: torch.Tensor) -> None:
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.numel() >= d
+    _check(lib().mlmc_aggregate_rtn(ctx, C.byref(msgs.struct), M, d, out.data_ptr(), _stream()), "mlmc_aggregate_rtn")
+
+
+class FloatBuffers:
+    """Caller-owned device buffers of a floating-point message batch."""
+
+    def __init__(self, M: int, d: int, w_max: int, device: str = "cuda"):
+        self.M, self.d, self.w_max = M, d, w_max
+        self.words = (d + 31) // 32
+        self.expo = torch.zeros((M, self.words * 32), dtype=torch.uint8, device=device)
+        self.planes = torch.zeros((M, 1 + w_max, self.words), dtype=torch.int32, device=device)  # uint32 payload
+        self.level = torch.full((M,), -1, dtype=torch.int32, device=device)
+        self.p_sel = torch.zeros(M, dtype=torch.float64, device=device)
+        self.struct = mlmc_float_msgs(self.expo.data_ptr(), self.planes.data_ptr(), self.level.data_ptr(),
+                                      self.p_sel.data_ptr(), w_max)
+
+
+class RtnBuffers:
+    """Caller-owned device buffers of a dense MLMC-RTN message batch (rows padded to 16 bytes)."""
+
+    def __init__(self, M: int, d: int, device: str = "cuda"):
+        self.M, self.d = M, d
+        self.ldv = (d + 3) // 4 * 4
+        self.val = torch.zeros((M, self.ldv), dtype=torch.float32, device=device)
+        self.c = torch.zeros(M, dtype=torch.float32, device=device)
+        self.level = torch.full((M,), -1, dtype=torch.int32, device=device)
+        self.p_sel = torch.zeros(M, dtype=torch.float64, device=device)
+        self.struct = mlmc_rtn_msgs(self.val.data_ptr(), self.c.data_ptr(), self.level.data_ptr(),
+                                    self.p_sel.data_ptr(), self.ldv)
 
 
 class TopkBuffers:

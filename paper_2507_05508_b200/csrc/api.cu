@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -69,6 +70,31 @@ int check_bit_schedule(const I* b, int L, int32_t* b32) {
         b32[l] = (int32_t)b[l];
     }
     return MLMC_OK;
+}
+
+// RTN widths r_0 < ... < r_{L-2} <= 16 (App. G); level L-1 is the identity and has no width.
+template <typename I>
+int check_rtn_schedule(const I* r, int L, int32_t* r32) {
+    if (L < 1 || L > 17) return MLMC_ERR_ARG;
+    if (L > 1 && !r) return MLMC_ERR_ARG;
+    int64_t prev = 0;
+    for (int l = 0; l + 1 < L; ++l) {
+        if (r[l] <= prev || r[l] > 16) return MLMC_ERR_SCHEDULE;
+        prev = r[l];
+        r32[l] = (int32_t)r[l];
+    }
+    return MLMC_OK;
+}
+
+// Mantissa digits mb_0 < ... < mb_{L-1} = F kept by the floating-point levels (App. B); the top level is the identity.
+int check_mantissa_schedule(const int32_t* mb, int L, int F) {
+    if (!mb) return MLMC_ERR_ARG;
+    int prev = 0;
+    for (int l = 0; l < L; ++l) {
+        if (mb[l] <= prev || mb[l] > F) return MLMC_ERR_SCHEDULE;
+        prev = mb[l];
+    }
+    return mb[L - 1] == F ? MLMC_OK : MLMC_ERR_SCHEDULE;
 }
 
 // Lemma 3.2 asks for non-zero probabilities; they are renormalised in fp64.
@@ -183,6 +209,12 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_gmax = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_S = pl.take(sizeof(unsigned long long) * kMaxLevels * ws.stat_ctas * M_max);
     const size_t o_blevel = pl.take(sizeof(int32_t) * M_max);
+    ws.big_cap = d_max < (int64_t(1) << 20) ? d_max : (int64_t(1) << 20);
+    const size_t o_pbig = pl.take(sizeof(double) * ws.big_cap);
+    const size_t o_cbig = pl.take(sizeof(double) * ws.big_cap);
+    ws.rtn_ctas = ws.sm_count * 8;
+    ws.cur_rtn_ctas = 0;
+    const size_t o_rtn = pl.take(sizeof(double) * kMaxLevels * ws.rtn_ctas * M_max);
 
     ctx->slab_bytes = pl.off;
     if (cudaMalloc(&ctx->slab, ctx->slab_bytes) != cudaSuccess) {
@@ -225,6 +257,9 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.gmax_bits = reinterpret_cast<uint32_t*>(base + o_gmax);
     ws.S_partial = reinterpret_cast<unsigned long long*>(base + o_S);
     ws.bit_level = reinterpret_cast<int32_t*>(base + o_blevel);
+    ws.p_big = reinterpret_cast<double*>(base + o_pbig);
+    ws.cdf_big = reinterpret_cast<double*>(base + o_cbig);
+    ws.rtn_partial = reinterpret_cast<double*>(base + o_rtn);
     if (cudaDeviceSynchronize() != cudaSuccess) {
         cudaFree(ctx->slab);
         delete ctx;
@@ -271,7 +306,8 @@ int64_t mlmc_launch_count(const mlmc_ctx* ctx) { return ctx ? ctx->ws.launches :
 static const char* const kKernelNames[K_COUNT] = {
     "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "sums_candidates", "cand_pass2", "masked_pass2",
     "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
-    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide", "reset"};
+    "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide", "reset",
+    "float_draw", "float_pack", "aggregate_floatbits", "rtn_stats", "rtn_probs_draw", "rtn_emit", "aggregate_dense", "stopk_draw", "stopk_params"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
 
@@ -338,14 +374,16 @@ int mlmc_level_probs(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, 
                      const int64_t* sched, int L, const double* p_host, double* p_out, double* delta_out,
                      void* stream) {
     if (int rc = check_common(ctx, g, dtype, d, M, ld, L)) return rc;
-    if (!p_out || (kind != MLMC_TOPK && kind != MLMC_BITWISE)) return MLMC_ERR_ARG;
+    if (!p_out || (kind != MLMC_TOPK && kind != MLMC_BITWISE && kind != MLMC_RTN)) return MLMC_ERR_ARG;
     Workspace& ws = ctx->ws;
     double pn[kMaxLevels];
     int32_t b32[kMaxLevels];
     if (kind == MLMC_TOPK) {
         if (int rc = check_topk_schedule(sched, L, d)) return rc;
-    } else {
+    } else if (kind == MLMC_BITWISE) {
         if (int rc = check_bit_schedule(sched, L, b32)) return rc;
+    } else {
+        if (int rc = check_rtn_schedule(sched, L, b32)) return rc;
     }
     if (p_host)
         if (int rc = normalise_probs(p_host, L, pn)) return rc;
@@ -362,11 +400,17 @@ int mlmc_level_probs(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, 
             run_band_norms(ws, g, dtype, d, M, ld, L, s);
             launch_probs_draw(ws, dtype, M, L, d, true, false, 0, 0, nullptr, s);
         }
-    } else {
+    } else if (kind == MLMC_BITWISE) {
         if (need_data) {
             launch_absmax(ws, g, dtype, d, M, ld, s);
             launch_bit_stats(ws, g, dtype, d, M, ld, b32, L, s);
             launch_bit_probs_draw(ws, M, b32, L, true, true, 0, 0, nullptr, s);
+        }
+    } else {
+        if (need_data) {
+            launch_absmax(ws, g, dtype, d, M, ld, s);
+            launch_rtn_stats(ws, g, dtype, d, M, ld, b32, L, s);
+            launch_rtn_probs_draw(ws, M, L, true, true, 0, 0, nullptr, s);
         }
     }
     launch_copy_probs(ws, M, L, p_host ? ws.p_fixed : nullptr, p_out, delta_out, s);
@@ -445,6 +489,125 @@ int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, 
     } else {
         return MLMC_ERR_ARG;
     }
+    return finish(cudaGetLastError());
+}
+
+int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int64_t s_len,
+                        const double* p, uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, void* stream) {
+    if (!ctx || s_len < 1 || d < 1) return MLMC_ERR_ARG;
+    const int64_t L = (d + s_len - 1) / s_len;
+    if (L <= kMaxLevels) {  // few segments: the general Top-k path with the uniform schedule k_l = min(d, s (l + 1))
+        int64_t k[kMaxLevels];
+        for (int64_t l = 0; l < L; ++l) k[l] = (s_len * (l + 1) < d) ? s_len * (l + 1) : d;
+        return mlmc_compress_topk(ctx, g, dtype, d, M, ld, k, (int)L, p, seed, step, out, stream);
+    }
+    if (int rc = check_common(ctx, g, dtype, d, M, ld, 1)) return rc;
+    if (!out || !out->idx || !out->val || !out->count || !out->level || !out->p_sel || out->capacity < 0)
+        return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    if (!p || L > ws.big_cap) return MLMC_ERR_ARG;  // adaptive p needs every segment norm: L <= MLMC_MAX_LEVELS only
+    // normalised p and its running sums in ascending l (the draw is min{ l : u < cdf_l }, the last cdf is 1)
+    std::vector<double> pn((size_t)L), cdf((size_t)L);
+    double sum = 0.0;
+    for (int64_t l = 0; l < L; ++l) {
+        if (!(p[l] > 0.0) || !std::isfinite(p[l])) return MLMC_ERR_PROB;
+        sum += p[l];
+    }
+    if (std::fabs(sum - 1.0) > 1e-9) return MLMC_ERR_PROB;
+    double c = 0.0;
+    for (int64_t l = 0; l < L; ++l) {
+        pn[(size_t)l] = p[l] / sum;
+        c += pn[(size_t)l];
+        cdf[(size_t)l] = (l == L - 1) ? 1.0 : c;
+    }
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+    cudaMemcpyAsync(ws.p_big, pn.data(), sizeof(double) * L, cudaMemcpyHostToDevice, s);
+    cudaMemcpyAsync(ws.cdf_big, cdf.data(), sizeof(double) * L, cudaMemcpyHostToDevice, s);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MLMC_ERR_CUDA;  // the host arrays go out of scope below
+    launch_stopk_draw(ws, M, L, s_len, d, seed, step, s);
+    run_selection(ws, g, dtype, d, M, ld, 3, false, s);  // two queries per worker
+    launch_stopk_params(ws, M, s_len, d, out, s);
+    launch_emit(ws, g, dtype, d, M, ld, *out, s);
+    return finish(cudaGetLastError());
+}
+
+int mlmc_compress_floatbits(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* mb,
+                            int L, const double* p, uint64_t seed, uint64_t step, const mlmc_float_msgs* out,
+                            void* stream) {
+    if (int rc = check_common(ctx, g, dtype, d, M, ld, L)) return rc;
+    if (!out || !out->expo || !out->planes || !out->level || !out->p_sel || out->w_max < 1) return MLMC_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(out->expo) % 16 != 0 || reinterpret_cast<uintptr_t>(out->planes) % 16 != 0)
+        return MLMC_ERR_ARG;
+    if (int rc = check_mantissa_schedule(mb, L, dtype == MLMC_BF16 ? 7 : 23)) return rc;
+    double pn[kMaxLevels];
+    if (p) {
+        if (int rc = normalise_probs(p, L, pn)) return rc;
+    } else {
+        // App. B's lemma: p^l proportional to 2^-l for the unit schedule; for a general schedule its worst-case
+        // argument gives p^l proportional to the largest residual of the level, 2^-mb_{l-1} - 2^-mb_l
+        double sum = 0.0;
+        for (int l = 0; l < L; ++l) {
+            pn[l] = std::ldexp(1.0, -(l ? mb[l - 1] : 0)) - std::ldexp(1.0, -mb[l]);
+            sum += pn[l];
+        }
+        for (int l = 0; l < L; ++l) pn[l] /= sum;
+    }
+    Workspace& ws = ctx->ws;
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+    cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
+    launch_compress_floatbits(ws, g, dtype, d, M, ld, mb, L, seed, step, *out, s);
+    return finish(cudaGetLastError());
+}
+
+int mlmc_aggregate_floatbits(mlmc_ctx* ctx, const mlmc_float_msgs* msgs, const int32_t* mb, int L, int M, int64_t d,
+                             float* out, void* stream) {
+    if (!ctx || !msgs || !out || !msgs->expo || !msgs->planes || !msgs->level || !msgs->p_sel) return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    if (d < 1 || d > ws.d_max || M < 1 || M > ws.M_max || L < 1 || L > kMaxLevels) return MLMC_ERR_ARG;
+    if (!mb) return MLMC_ERR_ARG;
+    int prev = 0;
+    for (int l = 0; l < L; ++l) {
+        if (mb[l] <= prev || mb[l] > 23) return MLMC_ERR_SCHEDULE;
+        prev = mb[l];
+    }
+    DeviceGuard guard(ws.device);
+    launch_aggregate_floatbits(ws, *msgs, mb, L, M, d, out, static_cast<cudaStream_t>(stream));
+    return finish(cudaGetLastError());
+}
+
+int mlmc_compress_rtn(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* r, int L,
+                      const double* p, uint64_t seed, uint64_t step, const mlmc_rtn_msgs* out, void* stream) {
+    if (int rc = check_common(ctx, g, dtype, d, M, ld, L)) return rc;
+    if (!out || !out->val || !out->c || !out->level || !out->p_sel || out->ldv < d) return MLMC_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(out->val) % 16 != 0) return MLMC_ERR_ARG;
+    int32_t r32[kMaxLevels] = {};
+    if (int rc = check_rtn_schedule(r, L, r32)) return rc;
+    double pn[kMaxLevels];
+    if (p)
+        if (int rc = normalise_probs(p, L, pn)) return rc;
+    Workspace& ws = ctx->ws;
+    DeviceGuard guard(ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+    const bool adaptive = (p == nullptr);
+    if (!adaptive) cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
+    launch_absmax(ws, g, dtype, d, M, ld, s);  // c = max |g|, and the NaN / Inf check
+    if (adaptive) launch_rtn_stats(ws, g, dtype, d, M, ld, r32, L, s);
+    launch_rtn_probs_draw(ws, M, L, adaptive, adaptive, seed, step, out, s);
+    launch_rtn_emit(ws, g, dtype, d, M, ld, r32, L, *out, s);
+    return finish(cudaGetLastError());
+}
+
+int mlmc_aggregate_rtn(mlmc_ctx* ctx, const mlmc_rtn_msgs* msgs, int M, int64_t d, float* out, void* stream) {
+    if (!ctx || !msgs || !out || !msgs->val || !msgs->level || msgs->ldv < d) return MLMC_ERR_ARG;
+    Workspace& ws = ctx->ws;
+    if (d < 1 || d > ws.d_max || M < 1 || M > ws.M_max) return MLMC_ERR_ARG;
+    DeviceGuard guard(ws.device);
+    launch_aggregate_dense(ws, msgs->val, msgs->level, M, d, msgs->ldv, out, static_cast<cudaStream_t>(stream));
     return finish(cudaGetLastError());
 }
 

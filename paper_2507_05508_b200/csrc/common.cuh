@@ -52,7 +52,8 @@ struct EmitParams {
 enum KernelId {
     K_DRAW_FIXED = 0, K_INIT_QUERIES, K_UNIFORMS, K_HIST1, K_RESOLVE1, K_SUMS_CAND, K_CAND2, K_MASKED2, K_RESOLVE2, K_CAND3,
     K_MASKED3, K_RESOLVE3, K_CAND_SUMS, K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
-    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_TILE_LIST, K_BAND_COUNT, K_BAND_SCAN, K_BIT_PACK_WIDE, K_RESET, K_COUNT
+    K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_TILE_LIST, K_BAND_COUNT, K_BAND_SCAN, K_BIT_PACK_WIDE, K_RESET,
+    K_FLOAT_DRAW, K_FLOAT_PACK, K_AGG_FLOAT, K_RTN_STATS, K_RTN_DRAW, K_RTN_EMIT, K_AGG_DENSE, K_STOPK_DRAW, K_STOPK_PARAMS, K_COUNT
 };
 
 constexpr int kTimingPool = 2048;  // event pairs kept between two reads
@@ -107,6 +108,13 @@ struct Workspace {
     unsigned long long* S_partial;  // [M][stat_ctas][kMaxLevels]
     int stat_ctas, cur_stat_ctas;
     int32_t* bit_level;          // [M] (mirrors out->level for the pack kernel)
+    // s-Top-k with more levels than kMaxLevels (fixed p only): normalised p and its running sums
+    double* p_big;               // [big_cap]
+    double* cdf_big;             // [big_cap]
+    int64_t big_cap;
+    // RTN: per-block residual energies of every level
+    double* rtn_partial;         // [M][rtn_ctas][kMaxLevels]
+    int rtn_ctas, cur_rtn_ctas;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -127,6 +135,21 @@ __device__ __forceinline__ double counter_uniform(uint64_t seed, uint64_t step, 
     h = splitmix_finalize(h + step + golden);
     h = splitmix_finalize(h + worker + golden);
     return (double)(h >> 11) * 0x1.0p-53;
+}
+
+// cdf in ascending l; the last level with p > 0 and everything after it has cdf 1; l* = min{l : u < cdf_l}
+// ("Sample l ~ p^l", Alg. 2 / Alg. 3).
+__device__ __forceinline__ int draw_from_probs(const double* p, int L, double u) {
+    int j_last = -1;
+    for (int j = 0; j < L; ++j)
+        if (p[j] > 0.0) j_last = j;
+    double c = 0.0;
+    for (int j = 0; j < L; ++j) {
+        c += p[j];
+        const double cdf = (j >= j_last) ? 1.0 : c;
+        if (u < cdf) return j;
+    }
+    return 0;
 }
 
 // Magnitude key: monotone in |g| for finite values.  fp32: 31 bits; bf16: 15 bits.
@@ -270,5 +293,24 @@ void launch_bit_pack(Workspace& ws, const void* g, int dtype, int64_t d, int M, 
                      const mlmc_bit_msgs& out, cudaStream_t s);
 void launch_aggregate_bitwise(Workspace& ws, const mlmc_bit_msgs& msgs, const int32_t* b, int L, int M, int64_t d,
                               float* out, cudaStream_t s);
+
+// floatbits.cu
+void launch_compress_floatbits(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* mb,
+                               int L, uint64_t seed, uint64_t step, const mlmc_float_msgs& out, cudaStream_t s);
+void launch_aggregate_floatbits(Workspace& ws, const mlmc_float_msgs& msgs, const int32_t* mb, int L, int M, int64_t d,
+                                float* out, cudaStream_t s);
+// rtn.cu
+void launch_rtn_stats(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* r, int L,
+                      cudaStream_t s);
+void launch_rtn_probs_draw(Workspace& ws, int M, int L, bool adaptive, bool have_stats, uint64_t seed, uint64_t step,
+                           const mlmc_rtn_msgs* out, cudaStream_t s);
+void launch_rtn_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, const int32_t* r, int L,
+                     const mlmc_rtn_msgs& out, cudaStream_t s);
+void launch_aggregate_dense(Workspace& ws, const float* val, const int32_t* level, int M, int64_t d, int64_t ldv,
+                            float* out, cudaStream_t s);
+// topk_select.cu: s-Top-k with many levels (fixed p)
+void launch_stopk_draw(Workspace& ws, int M, int64_t L, int64_t s_len, int64_t d, uint64_t seed, uint64_t step,
+                       cudaStream_t s);
+void launch_stopk_params(Workspace& ws, int M, int64_t s_len, int64_t d, const mlmc_topk_msgs* out, cudaStream_t s);
 
 }  // namespace mlmc

@@ -873,6 +873,60 @@ __global__ void copy_probs_kernel(const double* p_all, const double* delta_all, 
     if (delta_out) delta_out[i] = bad ? 0.0 : delta_all[m * kMaxLevels + l];
 }
 
+// -------------------------------------------------------------------------------------------
+// s-Top-k with more levels than kMaxLevels (fixed p): the level is drawn first, and the two ranks that bound its
+// segment, s l and min(d, s (l + 1)), are the only queries (Sec. 3.2: the residual is the l-th segment)
+// -------------------------------------------------------------------------------------------
+__global__ void stopk_draw_kernel(const double* __restrict__ p_big, const double* __restrict__ cdf_big, int64_t L,
+                                  int64_t s_len, int64_t d, uint64_t seed, uint64_t step, int M, double* p_all,
+                                  double* u_dev, EmitParams* emit, Query* queries) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= M) return;
+    const double u = counter_uniform(seed, step, (uint64_t)m);
+    u_dev[m] = u;
+    int64_t lo = 0, hi = L - 1;  // l* = min{ l : u < cdf_l }; the running sums are nondecreasing and end at 1 > u
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (u < cdf_big[mid]) hi = mid; else lo = mid + 1;
+    }
+    emit[m].level = (int32_t)lo;
+    p_all[m * kMaxLevels] = p_big[lo];
+    const int64_t kk[2] = {s_len * lo, min(d, s_len * (lo + 1))};
+    for (int j = 0; j < 2; ++j) {
+        Query q = {};
+        q.k = (uint32_t)kk[j];
+        q.slot = kNoSlot;
+        q.trivial = (kk[j] <= 0) ? 1u : (kk[j] >= d ? 2u : 0u);
+        if (q.trivial == 1u) {
+            q.T = kKeyNone;
+        } else if (q.trivial == 2u) {
+            q.T = 0u;
+            q.r = 0xFFFFFFFFu;
+        }
+        queries[m * kMaxQueries + j] = q;
+    }
+}
+
+__global__ void stopk_params_kernel(const Query* queries, int64_t s_len, int64_t d, const double* p_all, EmitParams* emit,
+                                    int64_t* out_count, int32_t* out_level, double* out_p_sel, int64_t capacity,
+                                    int* status, int* worker_err, int M) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= M) return;
+    if (worker_err[m]) {
+        fail_worker(m, emit, out_count, out_level, out_p_sel);
+        return;
+    }
+    const int32_t level = emit[m].level;
+    // the segment as the middle band of the three-level schedule (s l, min(d, s (l + 1)), d)
+    const int64_t k3[3] = {s_len * level, min(d, s_len * ((int64_t)level + 1)), d};
+    fill_emit(m, 1, p_all[m * kMaxLevels], queries + m * kMaxQueries, k3, 3, d, emit, out_count, out_level, out_p_sel,
+              capacity, status, worker_err);
+    if (emit[m].enabled) {
+        emit[m].level = level;
+        out_level[m] = level;
+    }
+}
+
 // Everything a selection accumulates into, cleared by one launch: the three histograms, the tile maxima, the
 // candidate counters and sums (zero), and the digit-2 slot map ("no slot").
 struct ResetList {
@@ -1080,6 +1134,19 @@ void launch_copy_probs(Workspace& ws, int M, int L, const double* p_fixed, doubl
     LaunchScope t(ws, K_COPY_PROBS, s);
     copy_probs_kernel<<<(M * L + 127) / 128, 128, 0, s>>>(ws.p_all, ws.delta_all, p_fixed, M, L, p_out, delta_out,
                                                           ws.worker_err);
+}
+
+void launch_stopk_draw(Workspace& ws, int M, int64_t L, int64_t s_len, int64_t d, uint64_t seed, uint64_t step,
+                       cudaStream_t s) {
+    LaunchScope t(ws, K_STOPK_DRAW, s);
+    stopk_draw_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.p_big, ws.cdf_big, L, s_len, d, seed, step, M, ws.p_all, ws.u_dev,
+                                                      ws.emit, ws.queries);
+}
+
+void launch_stopk_params(Workspace& ws, int M, int64_t s_len, int64_t d, const mlmc_topk_msgs* out, cudaStream_t s) {
+    LaunchScope t(ws, K_STOPK_PARAMS, s);
+    stopk_params_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.queries, s_len, d, ws.p_all, ws.emit, out->count, out->level,
+                                                        out->p_sel, out->capacity, ws.status, ws.worker_err, M);
 }
 
 int configure_select_kernels() {
