@@ -53,7 +53,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c5a", "c5b"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c5a", "c5b", "c5f", "c5r", "c3s"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -195,11 +195,21 @@ class Runner:
             if x.kind == "topk":
                 sched = wl.topk_schedule(x)
                 msgs = B.TopkBuffers(x.M, wl.max_band(sched), self.dev)
+            elif x.kind == "stopk":
+                sched = list(range(-(-x.d // x.seg_len)))           # one entry per level (segment)
+                msgs = B.TopkBuffers(x.M, x.seg_len, self.dev)
+            elif x.kind == "rtn":
+                sched = list(x.bits) + [0]                          # the widths and the identity level
+                msgs = B.RtnBuffers(x.M, x.d, self.dev)
+            elif x.kind == "floatbits":
+                sched = list(x.bits)
+                widths = [sched[0]] + [sched[i] - sched[i - 1] for i in range(1, len(sched))]
+                msgs = B.FloatBuffers(x.M, x.d, max(widths), self.dev)
             else:
                 sched = list(x.bits)
                 widths = [sched[0]] + [sched[i] - sched[i - 1] for i in range(1, len(sched))]
                 msgs = B.BitBuffers(x.M, x.d, max(widths), self.dev)
-            p = None if x.adaptive else list(wl.geometric_probs(len(sched)))
+            p = None if (x.adaptive or x.kind == "floatbits") else list(wl.geometric_probs(len(sched)))
             self.plan.append((x, sched, p, msgs))
         self.L = [len(pl[1]) for pl in self.plan]
         torch.cuda.synchronize()
@@ -211,6 +221,15 @@ class Runner:
             if x.kind == "topk":
                 B.mlmc_compress_topk(self.ctx, g, sched, p, x.seed, i, msgs)
                 B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, self.dense)
+            elif x.kind == "stopk":
+                B.mlmc_compress_stopk(self.ctx, g, x.seg_len, p, x.seed, i, msgs)
+                B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, self.dense)
+            elif x.kind == "rtn":
+                B.mlmc_compress_rtn(self.ctx, g, sched[:-1], p, x.seed, i, msgs)
+                B.mlmc_aggregate_rtn(self.ctx, msgs, x.M, x.d, self.dense)
+            elif x.kind == "floatbits":
+                B.mlmc_compress_floatbits(self.ctx, g, sched, p, x.seed, i, msgs)
+                B.mlmc_aggregate_floatbits(self.ctx, msgs, sched, x.M, x.d, self.dense)
             else:
                 B.mlmc_compress_bitwise(self.ctx, g, sched, p, x.seed, i, msgs)
                 B.mlmc_aggregate(self.ctx, B.MLMC_BITWISE, msgs, sched, x.M, x.d, self.dense)
@@ -219,8 +238,13 @@ class Runner:
         """Per variant kind: bytes of the messages of the last step (written once by compress, read once by aggregate)."""
         out = {}
         for x, sched, p, msgs in self.plan:
-            if x.kind == "topk":
+            if x.kind in ("topk", "stopk"):
                 out["topk"] = float(msgs.count.sum().item()) * 8.0
+            elif x.kind == "rtn":
+                out["dense"] = float(sum(1 for l in msgs.level.tolist() if l >= 0)) * x.d * 4.0
+            elif x.kind == "floatbits":
+                widths = [sched[0]] + [sched[i] - sched[i - 1] for i in range(1, len(sched))]
+                out["floatbits"] = float(sum((1 + widths[l]) * msgs.words * 4 + x.d for l in msgs.level.tolist() if l >= 0))
             else:
                 widths = [sched[0]] + [sched[i] - sched[i - 1] for i in range(1, len(sched))]
                 out["bitwise"] = float(sum((1 + widths[l]) * msgs.words * 4 for l in msgs.level.tolist() if l >= 0))
@@ -236,12 +260,14 @@ def sweeps_charged(w, emit_read_frac=None) -> float:
     the kernels moved where that is less.  Top-k moves one whole histogram sweep, for adaptive fp32 a second whole
     sweep, and two passes over the listed tiles (emit_read_frac of the row each); the fixed-p candidate sweep,
     which also skips tiles, is counted as nothing, so the figure is a lower bound of the bytes moved."""
-    if w.kind == "topk":
+    if w.kind in ("topk", "stopk"):
         if emit_read_frac is None:
             return 2.0
         moved = 1.0 + (1.0 if (w.adaptive and w.dtype != "bf16") else 0.0) + 2.0 * emit_read_frac
         return min(2.0, moved)
-    return 3.0 if w.adaptive else 2.0
+    if w.kind == "floatbits":
+        return 1.0  # App. B's probabilities are fixed: the level is drawn before the data is read, one sweep packs it
+    return 3.0 if w.adaptive else 2.0  # bit-wise and RTN: max -> level statistics -> message
 
 
 # Algorithmic bytes of one launch of each kernel, as a function of (sweep bytes, message bytes of its variant, dense
@@ -250,12 +276,15 @@ def sweeps_charged(w, emit_read_frac=None) -> float:
 # read back, so its bytes are unknown (None) there.
 def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float, read_frac, adaptive: bool):
     mt, mb = msg.get("topk", 0.0), msg.get("bitwise", 0.0)
+    mf, md = msg.get("floatbits", 0.0), msg.get("dense", 0.0)
     listed = None if read_frac is None else read_frac * sweep
     table = {
         "hist1": sweep, "sums_candidates": sweep if adaptive else None, "masked_pass2": sweep, "masked_pass3": sweep,
         "norm_sweep": sweep, "band_count": listed, "emit": None if listed is None else listed + mt,
         "aggregate_topk": mt + dense,
         "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + mb, "aggregate_bitwise": mb + dense,
+        "float_pack": sweep + mf, "aggregate_floatbits": mf + dense,
+        "rtn_stats": sweep, "rtn_emit": sweep + md, "aggregate_dense": md + dense,
     }
     return table.get(name)
 
@@ -336,7 +365,7 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
             acc[1] += n
         for kind, v in r.message_bytes().items():
             msg_acc[kind] = msg_acc.get(kind, 0.0) + v
-        if any(x.kind == "topk" for x in subs):
+        if any(x.kind in ("topk", "stopk") for x in subs):
             listed, tiles = B.mlmc_read_listed_tiles(r.ctx, w.M)
             listed_acc += sum(listed) / float(max(1, tiles * w.M))
             listed_n += 1
@@ -347,7 +376,7 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
 
     # ---- roofline of the dominant kernel and of the whole step
     ratios = ncu_traffic_ratios()
-    adaptive_topk = any(x.kind == "topk" and x.adaptive for x in subs)
+    adaptive_topk = any(x.kind in ("topk", "stopk") and x.adaptive for x in subs)
     kernels = {}
     t_all = sum(v[0] for v in per_kernel.values())
     for name, (ms, n) in sorted(per_kernel.items(), key=lambda kv: -kv[1][0]):
@@ -485,6 +514,17 @@ def oracle_sample_step(subs, g_row_np, d_s: int, step: int):
             p = None if w.adaptive else wl.geometric_probs(len(k))
             m = oracle.topk(x, k, p=p, seed=w.seed, step=step, worker=0)
             oracle.aggregate_topk([(m.idx, m.val)], d_s)
+        elif w.kind == "stopk":
+            s_len = max(1, min(w.seg_len, d_s))
+            L = -(-d_s // s_len)
+            m = oracle.stopk(x, s_len, p=wl.geometric_probs(L), seed=w.seed, step=step, worker=0)
+            oracle.aggregate_topk([(m.idx, m.val)], d_s)
+        elif w.kind == "rtn":
+            m = oracle.rtn(x, list(w.bits), p=None, seed=w.seed, step=step, worker=0)
+            oracle.aggregate_dense([m.val], d_s)
+        elif w.kind == "floatbits":
+            m = oracle.floatbits(x, list(w.bits), p=None, seed=w.seed, step=step, worker=0)
+            oracle.aggregate_dense([m.est], d_s)
         else:
             b = list(w.bits)
             p = None if w.adaptive else wl.geometric_probs(len(b))

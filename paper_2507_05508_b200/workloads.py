@@ -26,7 +26,7 @@ import torch
 @dataclass(frozen=True)
 class Workload:
     name: str
-    kind: str                 # "topk" | "bitwise"
+    kind: str                 # "topk" | "bitwise" | "floatbits" | "rtn" | "stopk"
     d: int
     M: int
     dtype: str                # "f32" | "bf16"
@@ -42,7 +42,8 @@ class Workload:
     outlier_mult: float = 1.0
     k_base: int = 0           # topk: k_l = k_base * 2^l            (when k_den == 0)
     k_den: int = 0            # topk: k_l = min(d, floor(d * 2^l / k_den))
-    bits: tuple = ()          # bitwise: b_l
+    bits: tuple = ()          # bitwise: b_l;  floatbits: mantissa digits mb_l;  rtn: widths r_l (identity level implied)
+    seg_len: int = 0          # stopk: segment length s
 
 
 C1 = Workload("c1", "topk", 65_536, 4, "f32", False, 0, 10, "normal", "coord_loguniform", 1e-3, 1.0, k_base=64)
@@ -56,7 +57,12 @@ C5A = Workload("c5a", "topk", 124_439_808, 8, "f32", True, 4, 10, "normal", "seg
                outlier_frac=1e-3, outlier_mult=100.0, k_den=10000)
 C5B = replace(C5A, name="c5b", kind="bitwise", k_den=0, bits=(1, 2, 4, 8, 16, 23))
 
-ALL = {w.name: w for w in (C1, C2, C3, C4, C5A, C5B)}
+# The further compressors of the paper on the same synthetic gradients (not BASELINE configs: measured beside them).
+C5F = replace(C5A, name="c5f", kind="floatbits", adaptive=False, k_den=0, bits=(1, 2, 4, 8, 16, 23))   # App. B, fixed p
+C5R = replace(C5A, name="c5r", kind="rtn", k_den=0, bits=(2, 4, 8, 16))                                # App. G, adaptive
+C3S = replace(C3, name="c3s", kind="stopk", k_den=0, seg_len=11_690)                                   # App. D, L = 1000, fixed p
+
+ALL = {w.name: w for w in (C1, C2, C3, C4, C5A, C5B, C5F, C5R, C3S)}
 
 
 def shrink(w: Workload, d: int, M: Optional[int] = None) -> Workload:
