@@ -1,6 +1,7 @@
 """Parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times.
 
-The oracle cannot sort eight 124M-entry rows in reasonable time, so per workload
+The oracle cannot sort eight 124M-entry rows in reasonable time, so per workload and for the first and the last step
+of the config
   * one worker's whole row goes through the oracle and is compared element by element
     (level, probability, every band index, every value; bit planes for the bit-wise path),
   * every worker is checked through properties that hold at any size: the message has exactly
@@ -80,29 +81,35 @@ def _topk_fullsize(B, ora, w, step, oracle_workers=(0,)):
         B.mlmc_destroy(ctx)
 
 
-def test_c3_full_size(B, ora):
-    _topk_fullsize(B, ora, wl.C3, step=0, oracle_workers=(0, 15))
+# Steps {0, last} of every config; the whole-row oracle comparison takes a worker or two per step (a 124M-entry row
+# costs the oracle's full sort about half a minute), every other worker goes through the properties above.
+@pytest.mark.parametrize("step,workers", [(0, (0, 15)), (wl.C3.steps - 1, (7,))])
+def test_c3_full_size(B, ora, step, workers):
+    _topk_fullsize(B, ora, wl.C3, step=step, oracle_workers=workers)
 
 
-def test_c4_full_size(B, ora):
-    _topk_fullsize(B, ora, wl.C4, step=1, oracle_workers=(31,))
+@pytest.mark.parametrize("step,workers", [(0, (0,)), (wl.C4.steps - 1, (31,))])
+def test_c4_full_size(B, ora, step, workers):
+    _topk_fullsize(B, ora, wl.C4, step=step, oracle_workers=workers)
 
 
-def test_c5a_full_size(B, ora):
-    _topk_fullsize(B, ora, wl.C5A, step=0, oracle_workers=(3,))
+@pytest.mark.parametrize("step,workers", [(0, (3,)), (wl.C5A.steps - 1, (6,))])
+def test_c5a_full_size(B, ora, step, workers):
+    _topk_fullsize(B, ora, wl.C5A, step=step, oracle_workers=workers)
 
 
-def test_c5b_full_size(B, ora):
+@pytest.mark.parametrize("step,workers", [(0, (0, 5)), (wl.C5B.steps - 1, (2,))])
+def test_c5b_full_size(B, ora, step, workers):
     w = wl.C5B
     torch.cuda.set_device(0)
     b = list(w.bits)
     widths = np.diff(np.concatenate([[0], b]))
     ctx = B.mlmc_create(0, w.d, w.M, 32)
     try:
-        g = wl.gradients(w, 0, "cuda")
+        g = wl.gradients(w, step, "cuda")
         out = B.BitBuffers(w.M, w.d, int(widths.max()))
         dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
-        B.mlmc_compress_bitwise(ctx, g, b, None, w.seed, 0, out)
+        B.mlmc_compress_bitwise(ctx, g, b, None, w.seed, step, out)
         B.mlmc_aggregate(ctx, B.MLMC_BITWISE, out, b, w.M, w.d, dense)
         assert B.mlmc_get_status(ctx) == B.MLMC_OK
         level, p_sel, gmax = out.level.tolist(), out.p_sel.tolist(), out.gmax.cpu().numpy()
@@ -118,11 +125,11 @@ def test_c5b_full_size(B, ora):
             mm.planes = out.planes[m, :1 + wv].cpu().numpy().view(np.uint32)
             mm.gmax, mm.level, mm.p_sel = float(gmax[m]), level[m], p_sel[m]
             msgs.append(mm)
-        for m in (0, 5):                                                   # whole rows through the oracle
+        for m in workers:                                                  # whole rows through the oracle
             row = wl.as_numpy_bits(g[m:m + 1])[0]
-            o = ora.bitwise(row, b, None, seed=w.seed, step=0, worker=m)
+            o = ora.bitwise(row, b, None, seed=w.seed, step=step, worker=m)
             if o.margin < MARGIN and level[m] != o.level:
-                o = ora.bitwise(row, b, None, seed=w.seed, step=0, worker=m, force_level=level[m])
+                o = ora.bitwise(row, b, None, seed=w.seed, step=step, worker=m, force_level=level[m])
             assert level[m] == o.level and np.float32(o.gmax) == gmax[m]
             assert abs(p_sel[m] - o.p_sel) <= 1e-10 * o.p_sel
             assert np.array_equal(msgs[m].planes, o.planes)

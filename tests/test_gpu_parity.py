@@ -322,6 +322,32 @@ def test_level_probs(B, ora, ctx):
         assert np.allclose(d_b[m].cpu().numpy(), o.delta, rtol=1e-13, atol=0)
 
 
+def test_level_probs_bf16(B, ora, ctx):
+    """mlmc_level_probs on bf16 input: Top-k (norms from the exact 2^15-bin counts) and bit-wise."""
+    w = wl.shrink(wl.C4, 500_009, 3)
+    k = wl.topk_schedule(w)
+    L = len(k)
+    g = padded(wl.gradients(w, 1, "cuda"), 8)
+    p_out = torch.zeros((3, L), dtype=torch.float64, device="cuda")
+    d_out = torch.zeros((3, L), dtype=torch.float64, device="cuda")
+    B.mlmc_level_probs(ctx, g, B.MLMC_TOPK, k, None, p_out, d_out)
+    assert B.mlmc_get_status(ctx) == 0
+    gh = wl.as_numpy_bits(g)
+    assert gh.dtype == np.uint16
+    for m in range(3):
+        o = ora.topk(gh[m], k, None)
+        assert np.allclose(p_out[m].cpu().numpy(), o.p, rtol=1e-11, atol=1e-15)
+        assert np.allclose(d_out[m].cpu().numpy(), o.delta, rtol=1e-12, atol=0)
+    b = [1, 2, 4, 8, 16, 23]
+    p_b = torch.zeros((3, 6), dtype=torch.float64, device="cuda")
+    d_b = torch.zeros((3, 6), dtype=torch.float64, device="cuda")
+    B.mlmc_level_probs(ctx, g, B.MLMC_BITWISE, b, None, p_b, d_b)
+    for m in range(3):
+        o = ora.bitwise(gh[m], b, None)
+        assert np.allclose(p_b[m].cpu().numpy(), o.p, rtol=1e-12, atol=1e-15)
+        assert np.allclose(d_b[m].cpu().numpy(), o.delta, rtol=1e-13, atol=0)
+
+
 def test_c2_bitwise_all_steps(B, ora, ctx):
     w = wl.C2
     b, p = list(w.bits), list(wl.geometric_probs(6))
