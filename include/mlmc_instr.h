@@ -38,6 +38,15 @@ int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_ho
  * Synchronous (copies from the device and waits for the stream); a measurement aid, not part of the method. */
 int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t* tiles_host, void* stream);
 
+/* Fixed-p Top-k on fp32 reuses, per worker and level boundary, the leading-digit bin in which the threshold was
+ * found by the last call on the same problem (same d, M, schedule, dtype) as a bracket: the first sweep collects the
+ * keys of that bin and its two neighbours, and when the new threshold bins fall inside, no second pass over the
+ * gradient is made for the candidates (Sec. 3, remark after Alg. 2: the residual without computing each term).
+ *   stats_host  host uint64[3], cumulative since mlmc_create: workers whose two brackets both held / workers with a
+ *               bracket that missed (the candidate pass ran) / workers without a stored bin yet.
+ * Synchronous; a measurement aid. */
+int mlmc_read_bracket_stats(mlmc_ctx* ctx, uint64_t* stats_host, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,6 +23,7 @@ MLMC_ERR_NONFINITE, MLMC_ERR_TIMEOUT, MLMC_ERR_CUDA, MLMC_ERR_NOMEM, MLMC_ERR_IN
 MLMC_MAX_LEVELS = 32
 
 EXPORTS = ["mlmc_create", "mlmc_destroy", "mlmc_get_status", "mlmc_launch_count", "mlmc_read_u", "mlmc_read_listed_tiles",
+           "mlmc_read_bracket_stats",
            "mlmc_kernel_count", "mlmc_kernel_name", "mlmc_timing_enable", "mlmc_timing_read",
            "mlmc_level_probs", "mlmc_compress_topk", "mlmc_compress_bitwise", "mlmc_aggregate",
            "mlmc_aggregate_topk_noalloc", "mlmc_compress_stopk", "mlmc_compress_floatbits", "mlmc_aggregate_floatbits",
@@ -74,6 +75,7 @@ def lib() -> C.CDLL:
         L.mlmc_launch_count.restype = i64
         L.mlmc_read_u.argtypes = [vp, u64, u64, i32, vp, vp]
         L.mlmc_read_listed_tiles.argtypes = [vp, i32, vp, vp, vp]
+        L.mlmc_read_bracket_stats.argtypes = [vp, vp, vp]
         L.mlmc_level_probs.argtypes = [vp, vp, i32, i64, i32, i64, i32, vp, i32, vp, vp, vp, vp]
         L.mlmc_compress_topk.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
         L.mlmc_compress_bitwise.argtypes = [vp, vp, i32, i64, i32, i64, vp, i32, vp, u64, u64, vp, vp]
@@ -169,6 +171,13 @@ def mlmc_read_listed_tiles(ctx, M: int):
     tiles = C.c_int64(0)
     _check(lib().mlmc_read_listed_tiles(ctx, M, buf, C.byref(tiles), _stream()), "mlmc_read_listed_tiles")
     return list(buf), int(tiles.value)
+
+
+def mlmc_read_bracket_stats(ctx):
+    """(workers whose brackets held, workers with a missed bracket, workers without a stored bin), cumulative."""
+    buf = (C.c_uint64 * 3)()
+    _check(lib().mlmc_read_bracket_stats(ctx, buf, _stream()), "mlmc_read_bracket_stats")
+    return tuple(int(x) for x in buf)
 
 
 def _g_args(g: torch.Tensor):

@@ -114,13 +114,16 @@ int finish(cudaError_t e) { return e == cudaSuccess ? MLMC_OK : MLMC_ERR_CUDA; }
 // Thresholds of every live query (sweep 1 + the two masked digit passes for fp32).
 // sweep 1 (leading-digit histogram), and for fp32 sweep 2 (candidates [+ energies]) and the two remaining
 // digit passes over the candidates.
+// brackets (fixed p, fp32): the first sweep also collects the keys of the bins around last call's boundary bins;
+// where both boundary bins of a worker's band fall inside, the candidate sweep has nothing left to do.
 void run_selection(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, int L, bool sums,
-                   cudaStream_t s) {
+                   bool brackets, cudaStream_t s) {
+    brackets = brackets && dtype == MLMC_F32 && !sums && L > 1;
     launch_reset_selection(ws, dtype, d, M, s);
-    launch_hist1(ws, g, dtype, d, M, ld, s);
-    launch_resolve1(ws, dtype, M, L, s);
+    launch_hist1(ws, g, dtype, d, M, ld, brackets, s);
+    launch_resolve1(ws, dtype, M, L, brackets, s);
     if (dtype == MLMC_F32) {
-        launch_sums_candidates(ws, g, d, M, ld, L, sums, s);
+        launch_sums_candidates(ws, g, d, M, ld, L, sums, brackets, s);
         if (L > 1) {
             launch_digit_pass(ws, g, d, M, ld, 2, s);
             launch_resolve23(ws, M, L, 2, s);
@@ -215,6 +218,12 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.rtn_ctas = ws.sm_count * 8;
     ws.cur_rtn_ctas = 0;
     const size_t o_rtn = pl.take(sizeof(double) * kMaxLevels * ws.rtn_ctas * M_max);
+    const size_t o_pbin = pl.take(sizeof(uint32_t) * kMaxLevels * M_max);
+    const size_t o_brk = pl.take(sizeof(uint4) * M_max);
+    const size_t o_bhit = pl.take(sizeof(int) * M_max);
+    const size_t o_bstat = pl.take(sizeof(unsigned long long) * 4);
+    ws.sig_d = ws.sig_ld = -1;
+    ws.sig_M = ws.sig_L = ws.sig_dtype = -1;
 
     ctx->slab_bytes = pl.off;
     if (cudaMalloc(&ctx->slab, ctx->slab_bytes) != cudaSuccess) {
@@ -260,6 +269,11 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.p_big = reinterpret_cast<double*>(base + o_pbig);
     ws.cdf_big = reinterpret_cast<double*>(base + o_cbig);
     ws.rtn_partial = reinterpret_cast<double*>(base + o_rtn);
+    ws.prev_bin = reinterpret_cast<uint32_t*>(base + o_pbin);
+    ws.bracket = reinterpret_cast<uint4*>(base + o_brk);
+    ws.bracket_hit = reinterpret_cast<int*>(base + o_bhit);
+    ws.bracket_stats = reinterpret_cast<unsigned long long*>(base + o_bstat);
+    cudaMemset(ws.prev_bin, 0xFF, sizeof(uint32_t) * kMaxLevels * M_max);
     if (cudaDeviceSynchronize() != cudaSuccess) {
         cudaFree(ctx->slab);
         delete ctx;
@@ -360,6 +374,15 @@ int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_ho
     return finish(cudaStreamSynchronize(s));
 }
 
+int mlmc_read_bracket_stats(mlmc_ctx* ctx, uint64_t* stats_host, void* stream) {
+    if (!ctx || !stats_host) return MLMC_ERR_ARG;
+    DeviceGuard guard(ctx->ws.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(stats_host, ctx->ws.bracket_stats, sizeof(uint64_t) * 3, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return MLMC_ERR_CUDA;
+    return finish(cudaStreamSynchronize(s));
+}
+
 int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t* tiles_host, void* stream) {
     if (!ctx || !listed_host || !tiles_host || M < 1 || M > ctx->ws.M_max) return MLMC_ERR_ARG;
     DeviceGuard guard(ctx->ws.device);
@@ -396,7 +419,7 @@ int mlmc_level_probs(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, 
         cudaMemcpyAsync(ws.k_dev, sched, sizeof(int64_t) * L, cudaMemcpyHostToDevice, s);
         if (need_data) {
             launch_init_queries_adaptive(ws, M, L, d, s);
-            run_selection(ws, g, dtype, d, M, ld, L, true, s);
+            run_selection(ws, g, dtype, d, M, ld, L, true, false, s);
             run_band_norms(ws, g, dtype, d, M, ld, L, s);
             launch_probs_draw(ws, dtype, M, L, d, true, false, 0, 0, nullptr, s);
         }
@@ -437,9 +460,17 @@ int mlmc_compress_topk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M
         launch_init_queries_adaptive(ws, M, L, d, s);
     } else {
         cudaMemcpyAsync(ws.p_fixed, pn, sizeof(double) * L, cudaMemcpyHostToDevice, s);
-        launch_draw_fixed(ws, M, L, d, seed, step, s);  // the draw does not depend on the data: only two thresholds are needed
+        // the bins stored by earlier calls belong to one problem: another shape or schedule starts afresh
+        bool same = ws.sig_d == d && ws.sig_ld == ld && ws.sig_M == M && ws.sig_L == L && ws.sig_dtype == dtype;
+        for (int l = 0; same && l < L; ++l) same = ws.sig_k[l] == k[l];
+        if (!same) {
+            cudaMemsetAsync(ws.prev_bin, 0xFF, sizeof(uint32_t) * kMaxLevels * ws.M_max, s);
+            ws.sig_d = d; ws.sig_ld = ld; ws.sig_M = M; ws.sig_L = L; ws.sig_dtype = dtype;
+            for (int l = 0; l < L; ++l) ws.sig_k[l] = k[l];
+        }
+        launch_draw_fixed(ws, M, L, d, seed, step, true, s);  // the draw does not depend on the data: only two thresholds are needed
     }
-    run_selection(ws, g, dtype, d, M, ld, L, adaptive, s);
+    run_selection(ws, g, dtype, d, M, ld, L, adaptive, !adaptive, s);
     if (adaptive) run_band_norms(ws, g, dtype, d, M, ld, L, s);
     launch_probs_draw(ws, dtype, M, L, d, adaptive, true, seed, step, out, s);
     launch_emit(ws, g, dtype, d, M, ld, *out, s);
@@ -527,7 +558,7 @@ int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int 
     cudaMemcpyAsync(ws.cdf_big, cdf.data(), sizeof(double) * L, cudaMemcpyHostToDevice, s);
     if (cudaStreamSynchronize(s) != cudaSuccess) return MLMC_ERR_CUDA;  // the host arrays go out of scope below
     launch_stopk_draw(ws, M, L, s_len, d, seed, step, s);
-    run_selection(ws, g, dtype, d, M, ld, 3, false, s);  // two queries per worker
+    run_selection(ws, g, dtype, d, M, ld, 3, false, false, s);  // two queries per worker
     launch_stopk_params(ws, M, s_len, d, out, s);
     launch_emit(ws, g, dtype, d, M, ld, *out, s);
     return finish(cudaGetLastError());

@@ -108,6 +108,14 @@ struct Workspace {
     unsigned long long* S_partial;  // [M][stat_ctas][kMaxLevels]
     int stat_ctas, cur_stat_ctas;
     int32_t* bit_level;          // [M] (mirrors out->level for the pack kernel)
+    // fixed-p Top-k: boundary bins of the previous call, per worker and level boundary, reused as brackets
+    uint32_t* prev_bin;          // [M][kMaxLevels] leading-digit bin of threshold j at the last call that resolved it (kKeyNone: none)
+    uint4* bracket;              // [M] {lo_a, width_a, lo_b, width_b}: bins collected as candidates by the first sweep
+    int* bracket_hit;            // [M] 1: both boundary bins of the drawn band lie in their brackets
+    unsigned long long* bracket_stats;  // [3] workers with both brackets hit / a bracket missed / no bracket yet (cumulative)
+    int64_t sig_d, sig_ld;       // host: the problem the stored bins belong to
+    int sig_M, sig_L, sig_dtype;
+    int64_t sig_k[kMaxLevels];
     // s-Top-k with more levels than kMaxLevels (fixed p only): normalised p and its running sums
     double* p_big;               // [big_cap]
     double* cdf_big;             // [big_cap]
@@ -262,13 +270,14 @@ struct LaunchScope {
 // topk_select.cu
 int configure_select_kernels();
 void launch_init_queries_adaptive(Workspace& ws, int M, int L, int64_t d, cudaStream_t s);
-void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, cudaStream_t s);
+void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, bool brackets,
+                       cudaStream_t s);
 void launch_uniforms(Workspace& ws, int M, uint64_t seed, uint64_t step, cudaStream_t s);
 void launch_reset_selection(Workspace& ws, int dtype, int64_t d, int M, cudaStream_t s);
-void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s);
-void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s);
+void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, bool brackets, cudaStream_t s);
+void launch_resolve1(Workspace& ws, int dtype, int M, int L, bool brackets, cudaStream_t s);
 void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,
-                            cudaStream_t s);
+                            bool brackets, cudaStream_t s);
 void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int pass, cudaStream_t s);
 void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s);
 void launch_band_norms_fp32(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, cudaStream_t s);

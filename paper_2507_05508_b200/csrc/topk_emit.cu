@@ -385,7 +385,7 @@ band_scan_kernel(uint4* __restrict__ rec, int tiles_per_worker, const uint32_t* 
 // position of a lane's first entry is the batch's base plus the entries of the lanes before it (one warp scan per
 // batch), and the lane then writes its own entries one after the other.
 template <typename T>
-__global__ void __launch_bounds__(kBandThreads)
+__global__ void __launch_bounds__(kBandThreads, 4)
 band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_worker,
                   const uint32_t* __restrict__ worker_tiles, const uint32_t* __restrict__ tile_n, int M,
                   const EmitParams* __restrict__ emit, const uint4* __restrict__ rec,

@@ -21,9 +21,24 @@ constexpr int kResolveThreads = 1024;
 // Adaptive: every level boundary k_0..k_{L-2} is a query.  Fixed p: the level is drawn first
 // (it does not depend on the data), and only the two boundaries of its band are live.
 __global__ void init_queries_kernel(Query* queries, const int64_t* k, int L, int64_t d, const EmitParams* emit,
-                                    int fixed) {
+                                    int fixed, const uint32_t* prev_bin, uint4* bracket) {
     const int m = blockIdx.x;
     const int j = threadIdx.x;
+    if (fixed && bracket && j == 0) {
+        // brackets of the first sweep: the bin where each boundary of the drawn band was found last time, and its
+        // two neighbours (an empty bracket is {lo = all ones, width = 0}: bin - lo wraps to bin + 1 > 0)
+        const int lv = emit[m].level;
+        uint4 b = make_uint4(0xFFFFFFFFu, 0u, 0xFFFFFFFFu, 0u);
+        if (lv >= 1) {
+            const uint32_t pb = prev_bin[m * kMaxLevels + lv - 1];
+            if (pb != kKeyNone) { b.x = pb ? pb - 1u : 0u; b.y = pb ? 2u : 1u; }
+        }
+        if (lv < L - 1) {
+            const uint32_t pb = prev_bin[m * kMaxLevels + lv];
+            if (pb != kKeyNone) { b.z = pb ? pb - 1u : 0u; b.w = pb ? 2u : 1u; }
+        }
+        bracket[m] = b;
+    }
     if (j >= L - 1) return;
     Query q = {};
     const int64_t kj = k[j];
@@ -78,13 +93,52 @@ __global__ void uniforms_kernel(double* u_dev, int M, uint64_t seed, uint64_t st
 // The sweep also records the largest key of every emit tile (kEmitTileVecs consecutive 16-byte vectors of the
 // row): the emit sweep reads only the tiles whose largest key reaches the lower threshold of the drawn band.
 // Chunks start at a multiple of 32 vectors, so the 32 vectors a warp loads together lie in one tile.
-template <typename T>
+// BR (fp32, fixed p): the keys whose leading digit lies in one of the worker's two brackets (the bins around last
+// call's boundary bins) are collected as candidates in the same sweep.  Every warp stages them in a private
+// shared-memory buffer, in lane order by a warp scan, and moves the buffer to the candidate list when it fills up
+// (one global counter update per move).
+constexpr int kWarpStage = 767;  // keys per warp stage (a warp adds at most 512 per trip), plus one word for its count: 96 KB per block
+
+template <typename T, bool BR>
 __global__ void __launch_bounds__(kHistThreads, 1)
 hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restrict__ hist1,
-             uint32_t* __restrict__ tile_max, int tiles_per_worker, int* status, int* worker_err) {
+             uint32_t* __restrict__ tile_max, int tiles_per_worker, int* status, int* worker_err,
+             const uint4* __restrict__ bracket, uint32_t* __restrict__ cand_keys, int64_t cand_cap,
+             uint32_t* cand_count, int* cand_overflow) {
     extern __shared__ uint32_t sh_hist[];
     using Tr = ElemTraits<T>;
     const int m = blockIdx.y;
+    // BR only: the warp's stage, its fill count in the word before it
+    uint32_t* wcount = sh_hist + kBins1 + (threadIdx.x >> 5) * (kWarpStage + 1);
+    uint32_t* wstage = wcount + 1;
+    uint32_t lo_a = 0xFFFFFFFFu, span_a = 0u, lo_b = 0xFFFFFFFFu, span_b = 0u;  // key ranges of the two brackets
+    if (BR) {
+        const uint4 br = bracket[m];
+        if (br.x != 0xFFFFFFFFu) { lo_a = br.x << 16; span_a = ((br.y + 1u) << 16) - 1u; }
+        if (br.z != 0xFFFFFFFFu) { lo_b = br.z << 16; span_b = ((br.w + 1u) << 16) - 1u; }
+        if ((threadIdx.x & 31) == 0) *wcount = 0u;
+    }
+    auto in_bracket = [&](uint32_t bits) -> bool {
+        const uint32_t key = bits & 0x7FFFFFFFu;
+        return (key - lo_a) <= span_a || (key - lo_b) <= span_b;  // an empty bracket: key - lo wraps to key + 1 > 0
+    };
+    auto flush_stage = [&]() {  // called by the whole warp, after a __syncwarp
+        const uint32_t wfill = *wcount;
+        if (wfill) {
+            uint32_t base = 0;
+            if ((threadIdx.x & 31) == 0) base = atomicAdd(&cand_count[m], wfill);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if ((int64_t)base + wfill <= cand_cap) {
+                uint32_t* dst = cand_keys + (int64_t)m * cand_cap + base;
+                for (uint32_t i = threadIdx.x & 31; i < wfill; i += 32) dst[i] = wstage[i];
+            } else if ((threadIdx.x & 31) == 0) {
+                cand_overflow[m] = 1;
+            }
+            __syncwarp();
+            if ((threadIdx.x & 31) == 0) *wcount = 0u;
+            __syncwarp();
+        }
+    };
     for (int b = threadIdx.x; b < kBins1; b += blockDim.x) sh_hist[b] = 0;
     __syncthreads();
     const T* row = g + (int64_t)m * ld;
@@ -116,6 +170,11 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
                 for_each_in_vector<T>(row, u, d, [&](int64_t, uint32_t bits) {
                     count_key(bits);
                     vm = max(vm, Tr::key(bits));
+                    if (BR && in_bracket(bits)) {  // the ragged end of the row: one by one
+                        const uint32_t at = atomicAdd(&cand_count[m], 1u);
+                        if ((int64_t)at < cand_cap) cand_keys[(int64_t)m * cand_cap + at] = bits & 0x7FFFFFFFu;
+                        else cand_overflow[m] = 1;
+                    }
                 });
                 bad |= vm >= Tr::kInfKey;
                 atomicMax(&tmax[u / kEmitTileVecs], vm);
@@ -137,6 +196,32 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
             bad |= wm >= Tr::kInfKey;  // a non-finite entry shows in the largest key of its warp
             if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitTileVecs], wm);
         }
+        if constexpr (BR) {
+            uint32_t cm = 0;  // bit 4 j + e: element e of vector j lies in a bracket
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                cm |= in_bracket(q[j].x) ? (1u << (4 * j)) : 0u;
+                cm |= in_bracket(q[j].y) ? (2u << (4 * j)) : 0u;
+                cm |= in_bracket(q[j].z) ? (4u << (4 * j)) : 0u;
+                cm |= in_bracket(q[j].w) ? (8u << (4 * j)) : 0u;
+            }
+            if (cm) {  // this lane's keys go to the warp's stage at a position taken from the warp's counter
+                uint32_t pos = atomicAdd(wcount, (uint32_t)__popc(cm));
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    if (cm & (1u << (4 * j))) wstage[pos++] = q[j].x & 0x7FFFFFFFu;
+                    if (cm & (2u << (4 * j))) wstage[pos++] = q[j].y & 0x7FFFFFFFu;
+                    if (cm & (4u << (4 * j))) wstage[pos++] = q[j].z & 0x7FFFFFFFu;
+                    if (cm & (8u << (4 * j))) wstage[pos++] = q[j].w & 0x7FFFFFFFu;
+                }
+            }
+            __syncwarp();
+            if (*wcount > (uint32_t)(kWarpStage - 32 * 4 * kBatch)) flush_stage();  // room for one more trip
+        }
+    }
+    if (BR) {
+        __syncwarp();
+        flush_stage();
     }
     if (bad) {
         worker_err[m] = MLMC_ERR_NONFINITE;
@@ -184,7 +269,8 @@ __device__ void assign_slots(Query* q, int nq, int shift) {
 // to its open interval  #{ j : bin_j > b }  (code < 64); a bin that holds one maps to 64 + its slot.
 __global__ void __launch_bounds__(kResolveThreads, 1)
 resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand_floor, int nq, int is_bf16,
-                const int* worker_err) {
+                const int* worker_err, const EmitParams* emit, const uint4* bracket, int* bracket_hit,
+                uint32_t* prev_bin, unsigned long long* bracket_stats, uint32_t* cand_count, int* cand_overflow) {
     __shared__ uint32_t sh_warp[32];
     __shared__ uint32_t sh_tot[kResolveThreads], sh_off[kResolveThreads];
     __shared__ int sh_bin[kMaxQueries];
@@ -270,6 +356,28 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand
         for (int j = 0; j < nq; ++j)
             if (sh_bin[j] >= 0 && sh_bin[j] < lowest) lowest = sh_bin[j];
         cand_floor[m] = (lowest < kBins1) ? ((uint32_t)lowest << 16) : 0xFFFFFFFFu;
+        if (bracket) {
+            // Did the first sweep already collect the keys of every boundary bin?  (fixed p: the live queries are
+            // the boundaries level - 1 and level of the drawn band.)  If not, its candidates are dropped and the
+            // candidate sweep runs.  Either way the bins are remembered for the next call.
+            const uint4 br = bracket[m];
+            const int lv = emit[m].level;
+            bool hit = cand_overflow[m] == 0, had = false;
+            for (int j = 0; j < nq; ++j) {
+                if (q[j].trivial) continue;
+                const uint32_t bin = (uint32_t)sh_bin[j];
+                const bool a = (j == lv - 1), inside = a ? (bin - br.x) <= br.y : (bin - br.z) <= br.w;
+                had |= (a ? br.x : br.z) != 0xFFFFFFFFu;
+                hit &= inside;
+                prev_bin[m * kMaxLevels + j] = bin;
+            }
+            bracket_hit[m] = hit ? 1 : 0;
+            if (!hit) {
+                cand_count[m] = 0u;
+                cand_overflow[m] = 0;
+            }
+            atomicAdd(&bracket_stats[hit ? 0 : (had ? 1 : 2)], 1ull);
+        }
     }
     uint8_t* tab = table1 + (int64_t)m * kBins1;
     for (int i = 0; i < per; ++i) {
@@ -304,7 +412,8 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
                        double* __restrict__ sum_partial, int sum_ctas,
                        uint32_t* __restrict__ cand_keys, int64_t cand_cap, uint32_t* cand_count, int* cand_overflow,
                        const int* worker_err, const uint32_t* __restrict__ tile_max,
-                       int tiles_per_worker, const uint32_t* __restrict__ cand_floor) {
+                       int tiles_per_worker, const uint32_t* __restrict__ cand_floor,
+                       const int* __restrict__ bracket_hit) {
     extern __shared__ __align__(16) uint8_t sh_raw[];
     uint8_t* sh_table = sh_raw;                                                   // [32768]
     uint32_t* sh_stage = reinterpret_cast<uint32_t*>(sh_raw + kBins1);            // [kStage]
@@ -313,6 +422,7 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
     __shared__ uint32_t sh_base;
     const int m = blockIdx.y;
     if (worker_err[m]) return;
+    if (!SUMS && bracket_hit && bracket_hit[m]) return;  // the first sweep collected every boundary-bin key already
     {
         const uint4* src = reinterpret_cast<const uint4*>(table + (int64_t)m * kBins1);
         uint4* dst = reinterpret_cast<uint4*>(sh_table);
@@ -366,7 +476,10 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
         if (threadIdx.x == 0) sh_n = 0;
         __syncthreads();
     };
-    auto take = [&](uint32_t bits) {
+    // One element: its energy goes to the interval's accumulator; a key of a boundary bin only sets its bit in `cm`,
+    // and the thread stages all its candidates of the round together (one counter update and one divergent region
+    // per thread and round instead of one per candidate).
+    auto take = [&](uint32_t bits, uint32_t bit, uint32_t& cm) {
         const uint32_t key = bits & 0x7FFFFFFFu;
         const uint32_t code = sh_table[key >> 16];
         if (code < 64u) {
@@ -376,7 +489,7 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
                 *a = fma(x, x, *a);
             }
         } else {
-            sh_stage[atomicAdd(&sh_n, 1u)] = key;
+            cm |= bit;
         }
     };
     auto load_round = [&](int64_t vb, uint4 (&q)[kS2Vecs]) {
@@ -399,13 +512,30 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
             for (int j = 0; j < kS2Vecs; ++j) cur[j] = nxt[j];
             continue;
         }
+        uint32_t cm = 0;  // bit 4 j + e: element e of vector j is a candidate
 #pragma unroll
         for (int j = 0; j < kS2Vecs; ++j) {
             const int64_t v = vb + j * kS2Threads + threadIdx.x;
             if (v < full_end) {
-                take(cur[j].x); take(cur[j].y); take(cur[j].z); take(cur[j].w);
-            } else if (v < v1) {  // ragged tail of the row
-                for (int64_t i = v * 4; i < d; ++i) take(reinterpret_cast<const uint32_t*>(row)[i]);
+                take(cur[j].x, 1u << (4 * j), cm); take(cur[j].y, 2u << (4 * j), cm);
+                take(cur[j].z, 4u << (4 * j), cm); take(cur[j].w, 8u << (4 * j), cm);
+            } else if (v < v1) {  // ragged tail of the row: staged one by one
+                for (int64_t i = v * 4; i < d; ++i) {
+                    uint32_t one = 0;
+                    const uint32_t bits = reinterpret_cast<const uint32_t*>(row)[i];
+                    take(bits, 1u, one);
+                    if (one) sh_stage[atomicAdd(&sh_n, 1u)] = bits & 0x7FFFFFFFu;
+                }
+            }
+        }
+        if (cm) {
+            uint32_t pos = atomicAdd(&sh_n, (uint32_t)__popc(cm));
+#pragma unroll
+            for (int j = 0; j < kS2Vecs; ++j) {
+                if (cm & (1u << (4 * j))) sh_stage[pos++] = cur[j].x & 0x7FFFFFFFu;
+                if (cm & (2u << (4 * j))) sh_stage[pos++] = cur[j].y & 0x7FFFFFFFu;
+                if (cm & (4u << (4 * j))) sh_stage[pos++] = cur[j].z & 0x7FFFFFFFu;
+                if (cm & (8u << (4 * j))) sh_stage[pos++] = cur[j].w & 0x7FFFFFFFu;
             }
         }
         __syncthreads();
@@ -445,7 +575,9 @@ cand_pass_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const
     const uint8_t* mp = map2 + (int64_t)m * kMaxQueries * kBins23;
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         const uint32_t key = cand[i];
-        const uint32_t s2 = (uint32_t)__ldg(&tab[key >> 16]) - 64u;
+        const uint32_t code = __ldg(&tab[key >> 16]);
+        if (code < 64u) continue;  // a bracket bin that holds no threshold after all
+        const uint32_t s2 = code - 64u;
         if (PASS == 2) {
             atomicAdd(&sh_hist[s2 * kBins23 + ((key >> 8) & 0xFFu)], 1u);
         } else {
@@ -963,18 +1095,20 @@ int blocks_per_worker(const Workspace& ws, int64_t d, int vec, int threads, int 
 void launch_init_queries_adaptive(Workspace& ws, int M, int L, int64_t d, cudaStream_t s) {
     if (L > 1) {
         LaunchScope t(ws, K_INIT_QUERIES, s);
-        init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 0);
+        init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 0, nullptr, nullptr);
     }
 }
 
-void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, cudaStream_t s) {
+void launch_draw_fixed(Workspace& ws, int M, int L, int64_t d, uint64_t seed, uint64_t step, bool brackets,
+                       cudaStream_t s) {
     {
         LaunchScope t(ws, K_DRAW_FIXED, s);
         draw_fixed_kernel<<<(M + 127) / 128, 128, 0, s>>>(ws.p_fixed, L, seed, step, ws.p_all, ws.u_dev, ws.emit, M);
     }
     if (L > 1) {
         LaunchScope t(ws, K_INIT_QUERIES, s);
-        init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 1);
+        init_queries_kernel<<<M, kMaxQueries, 0, s>>>(ws.queries, ws.k_dev, L, d, ws.emit, 1, ws.prev_bin,
+                                                      brackets ? ws.bracket : nullptr);
     }
 }
 
@@ -1007,25 +1141,34 @@ void launch_reset_selection(Workspace& ws, int dtype, int64_t d, int M, cudaStre
     reset_state_kernel<<<ws.sm_count * 2, 512, 0, s>>>(r);
 }
 
-void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, cudaStream_t s) {
+void launch_hist1(Workspace& ws, const void* g, int dtype, int64_t d, int M, int64_t ld, bool brackets, cudaStream_t s) {
     const int tpw = emit_tiles_per_worker(d, dtype);
     const size_t smem = kBins1 * sizeof(uint32_t);
     LaunchScope t(ws, K_HIST1, s);
     if (dtype == MLMC_BF16) {
         const int nb = blocks_per_worker(ws, d, 8, kHistThreads, M, 2);
-        hist1_kernel<bf16_t><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const bf16_t*>(g), d, ld, ws.hist1,
-                                                                     ws.tile_max, tpw, ws.status, ws.worker_err);
+        hist1_kernel<bf16_t, false><<<dim3(nb, M), kHistThreads, smem, s>>>(
+            static_cast<const bf16_t*>(g), d, ld, ws.hist1, ws.tile_max, tpw, ws.status, ws.worker_err, nullptr, nullptr, 0,
+            nullptr, nullptr);
     } else {
         const int nb = blocks_per_worker(ws, d, 4, kHistThreads, M, 2);
-        hist1_kernel<float><<<dim3(nb, M), kHistThreads, smem, s>>>(static_cast<const float*>(g), d, ld, ws.hist1,
-                                                                    ws.tile_max, tpw, ws.status, ws.worker_err);
+        if (brackets)
+            hist1_kernel<float, true><<<dim3(nb, M), kHistThreads, smem + (kHistThreads / 32) * (kWarpStage + 1) * sizeof(uint32_t), s>>>(
+                static_cast<const float*>(g), d, ld, ws.hist1, ws.tile_max, tpw, ws.status, ws.worker_err, ws.bracket,
+                ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow);
+        else
+            hist1_kernel<float, false><<<dim3(nb, M), kHistThreads, smem, s>>>(
+                static_cast<const float*>(g), d, ld, ws.hist1, ws.tile_max, tpw, ws.status, ws.worker_err, nullptr, nullptr,
+                0, nullptr, nullptr);
     }
 }
 
-void launch_resolve1(Workspace& ws, int dtype, int M, int L, cudaStream_t s) {
+void launch_resolve1(Workspace& ws, int dtype, int M, int L, bool brackets, cudaStream_t s) {
     LaunchScope t(ws, K_RESOLVE1, s);
     resolve1_kernel<<<M, kResolveThreads, 0, s>>>(ws.hist1, ws.queries, ws.table1, ws.cand_floor, L - 1,
-                                                  dtype == MLMC_BF16, ws.worker_err);
+                                                  dtype == MLMC_BF16, ws.worker_err, ws.emit,
+                                                  brackets ? ws.bracket : nullptr, ws.bracket_hit, ws.prev_bin,
+                                                  ws.bracket_stats, ws.cand_count, ws.cand_overflow);
 }
 
 static int cand_blocks(const Workspace& ws, int M) {
@@ -1039,7 +1182,7 @@ static size_t s2_smem(int L, bool sums) {
 
 // Sweep 2: energies of the threshold-free bins (adaptive only) and the candidate keys of the boundary bins.
 void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int64_t ld, int L, bool sums,
-                            cudaStream_t s) {
+                            bool brackets, cudaStream_t s) {
     int nb = blocks_per_worker(ws, d, 4, kS2Threads, M, sums ? 2 : 8);  // without the accumulators four blocks fit an SM
     if (nb > ws.sum_ctas) nb = ws.sum_ctas;
     ws.cur_sum_ctas = nb;
@@ -1049,12 +1192,12 @@ void launch_sums_candidates(Workspace& ws, const void* g, int64_t d, int M, int6
         sums_candidates_kernel<true><<<dim3(nb, M), kS2Threads, smem, s>>>(
             static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys,
             ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, ws.tile_max,
-            emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor);
+            emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor, nullptr);
     else
         sums_candidates_kernel<false><<<dim3(nb, M), kS2Threads, smem, s>>>(
             static_cast<const float*>(g), d, ld, ws.table1, L, ws.sum_partial, ws.sum_ctas, ws.cand_keys,
             ws.cand_cap, ws.cand_count, ws.cand_overflow, ws.worker_err, ws.tile_max,
-            emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor);
+            emit_tiles_per_worker(d, MLMC_F32), ws.cand_floor, brackets ? ws.bracket_hit : nullptr);
 }
 
 // Digit pass 2 or 3: over the candidate keys, and (early exit unless the buffer overflowed) over the full row.
@@ -1150,10 +1293,13 @@ void launch_stopk_params(Workspace& ws, int M, int64_t s_len, int64_t d, const m
 }
 
 int configure_select_kernels() {
-    cudaError_t e = cudaFuncSetAttribute(hist1_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(hist1_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(kBins1 * sizeof(uint32_t)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
-    e = cudaFuncSetAttribute(hist1_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(hist1_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kBins1 * sizeof(uint32_t) + (kHistThreads / 32) * (kWarpStage + 1) * sizeof(uint32_t)));
+    if (e != cudaSuccess) return MLMC_ERR_CUDA;
+    e = cudaFuncSetAttribute(hist1_kernel<bf16_t, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kBins1 * sizeof(uint32_t)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     const int smem_masked = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;

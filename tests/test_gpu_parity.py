@@ -227,6 +227,47 @@ def test_topk_candidate_overflow_takes_the_full_sweep_path(B, ora, ctx):
         check_topk(B, ora, ctx, g, k, list(wl.geometric_probs(len(k))), 11, step)
 
 
+def test_fixed_p_brackets_hit_miss_and_restart(B, ora):
+    """Fixed-p Top-k on fp32 reuses last call's boundary bins as brackets for the first sweep.  Every call must match
+    the oracle whether the brackets hold (same distribution, next step), miss (the gradient is rescaled: the candidate
+    pass runs after all) or do not exist yet (first call, new schedule)."""
+    w = wl.shrink(wl.C3, 400_003, 3)
+    k = wl.topk_schedule(w)
+    L = len(k)
+    c = B.mlmc_create(0, w.d, w.M, 32)
+    try:
+        sc = wl.scales(w, "cuda")
+        one_level = np.full(L, 1e-9)
+        one_level[3] = 1.0 - 1e-9 * (L - 1)                 # always level 3: the same two boundaries every step
+        p = list(one_level)
+        assert B.mlmc_read_bracket_stats(c) == (0, 0, 0)
+        g0 = padded(wl.gradients(w, 0, "cuda", sc), 4)
+        check_topk(B, ora, c, g0, k, p, w.seed, 0)
+        assert B.mlmc_read_bracket_stats(c) == (0, 0, 3)    # first call: nothing stored yet
+        for step in (1, 2, 3):
+            g = padded(wl.gradients(w, step, "cuda", sc), 4)
+            check_topk(B, ora, c, g, k, p, w.seed, step)
+        hit, miss, none = B.mlmc_read_bracket_stats(c)
+        assert none == 3 and hit + miss == 9 and hit >= 6   # fresh noise, same scales: the thresholds barely move
+        g_big = padded(wl.gradients(w, 4, "cuda", sc) * 1000.0, 4)
+        check_topk(B, ora, c, g_big, k, p, w.seed, 4)       # every threshold moved by ten binades: all brackets miss
+        hit2, miss2, none2 = B.mlmc_read_bracket_stats(c)
+        assert (hit2, miss2, none2) == (hit, miss + 3, none)
+        check_topk(B, ora, c, g_big, k, p, w.seed, 5)       # and hold again on the rescaled gradient
+        assert B.mlmc_read_bracket_stats(c)[0] == hit + 3
+        k2 = list(k)
+        k2[2] += 1                                          # another schedule: the stored bins are dropped
+        check_topk(B, ora, c, g_big, k2, p, w.seed, 6)
+        assert B.mlmc_read_bracket_stats(c)[2] == none + 3
+        check_topk(B, ora, c, g0, k, list(wl.geometric_probs(L)), w.seed, 7)    # mixed levels, partly known
+        check_topk(B, ora, c, g0, k, list(wl.geometric_probs(L)), w.seed, 8)
+        ties = to_dev(np.random.default_rng(3).choice(np.array([0.5, -0.5, 0.25, 3.0], dtype=np.float32), (3, w.d)))
+        check_topk(B, ora, c, ties, k, p, w.seed, 9)        # every key in two bins: brackets collect the whole row
+        check_topk(B, ora, c, ties, k, p, w.seed, 10)
+    finally:
+        B.mlmc_destroy(c)
+
+
 def test_topk_single_level_is_identity(B, ora, ctx):
     g_np = np.random.default_rng(23).standard_normal((3, 4097)).astype(np.float32)
     g = to_dev(g_np)
