@@ -279,8 +279,10 @@ def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float, read_frac
     mf, md = msg.get("floatbits", 0.0), msg.get("dense", 0.0)
     listed = None if read_frac is None else read_frac * sweep
     table = {
-        "hist1": sweep, "sums_candidates": sweep if adaptive else None, "masked_pass2": sweep, "masked_pass3": sweep,
-        "norm_sweep": sweep, "band_count": listed, "emit": None if listed is None else listed + mt,
+        # masked_pass2/3 and norm_sweep are the full-sweep fall-back of a worker whose candidates overflowed: they exit
+        # at once otherwise, so no bytes are claimed for them
+        "hist1": sweep, "sums_candidates": sweep if adaptive else None,
+        "band_count": listed, "emit": None if listed is None else listed + mt,
         "aggregate_topk": mt + dense,
         "absmax": sweep, "bit_stats": sweep, "bit_pack": sweep + mb, "aggregate_bitwise": mb + dense,
         "float_pack": sweep + mf, "aggregate_floatbits": mf + dense,

@@ -249,7 +249,8 @@ __device__ __forceinline__ int worker_of(const uint32_t* sh_off, int M, uint32_t
 
 // The tiles of every worker that can hold band entries, ascending: a tile whose largest key is below the lower
 // threshold Tb of the drawn band holds none (and no tie of Tb either), so the sweep leaves it out.
-// One block per worker; every thread owns a contiguous chunk of the tiles.
+// One block per worker; every warp owns a contiguous range of tiles (a multiple of 32, so that its rows of 32 tiles
+// are coalesced loads), counts its listed tiles, and after one barrier writes them behind those of the warps before.
 constexpr int kListThreads = 1024;
 
 __global__ void __launch_bounds__(kListThreads)
@@ -262,22 +263,19 @@ tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, co
     const uint32_t Tb = min(e.Tb, key_cap);
     const uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker;
     uint32_t* list = worker_tiles + (int64_t)m * tiles_per_worker;
-    const int per = (tiles_per_worker + kListThreads - 1) / kListThreads;
-    const int t0 = min((int)threadIdx.x * per, tiles_per_worker), t1 = min(t0 + per, tiles_per_worker);
-    uint32_t mine = 0;
-    if (on) {
-#pragma unroll 8
-        for (int t = t0; t < t1; ++t) mine += (__ldg(&tmax[t]) >= Tb) ? 1u : 0u;
-    }
-    // exclusive prefix over the threads
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += y;
+    const int rows = (tiles_per_worker + kListThreads - 1) / kListThreads;  // rows of 32 tiles per warp
+    const int t0 = warp * rows * 32;
+    uint32_t mine = 0;  // listed tiles of this warp (the same in every lane)
+    if (on) {
+#pragma unroll 4
+        for (int r = 0; r < rows; ++r) {
+            const int t = t0 + r * 32 + lane;
+            const bool f = t < tiles_per_worker && __ldg(&tmax[t]) >= Tb;
+            mine += __popc(__ballot_sync(0xFFFFFFFFu, f));
+        }
     }
-    if (lane == 31) sh_warp[warp] = incl;
+    if (lane == 0) sh_warp[warp] = mine;
     __syncthreads();
     uint32_t before = 0, total = 0;
     for (int w = 0; w < kListThreads / 32; ++w) {
@@ -285,11 +283,17 @@ tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, co
         total += x;
         if (w < warp) before += x;
     }
-    uint32_t pos = before + incl - mine;
-    if (on) {
-#pragma unroll 8
-        for (int t = t0; t < t1; ++t)
-            if (__ldg(&tmax[t]) >= Tb) list[pos++] = (uint32_t)t;
+    if (on && mine) {
+        uint32_t pos = before;
+        const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll 4
+        for (int r = 0; r < rows; ++r) {
+            const int t = t0 + r * 32 + lane;
+            const bool f = t < tiles_per_worker && __ldg(&tmax[t]) >= Tb;
+            const uint32_t mk = __ballot_sync(0xFFFFFFFFu, f);
+            if (f) list[pos + __popc(mk & lt)] = (uint32_t)t;
+            pos += __popc(mk);
+        }
     }
     if (threadIdx.x == 0) {
         tile_n[m] = total;
@@ -336,7 +340,9 @@ band_count_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
 }
 
 // Pass 2: exclusive running totals over the listed tiles of every worker, in place, and the self-check that the
-// band has exactly k_l - k_{l-1} entries.  One block per worker; every thread owns a contiguous chunk.
+// band has exactly k_l - k_{l-1} entries.  One block per worker; every warp owns a contiguous range of the list (a
+// multiple of 32 records, read as coalesced rows), adds it up, and after one barrier scans it row by row from the
+// total of the warps before it.
 __global__ void __launch_bounds__(kListThreads)
 band_scan_kernel(uint4* __restrict__ rec, int tiles_per_worker, const uint32_t* __restrict__ tile_n,
                  const EmitParams* __restrict__ emit, int* status) {
@@ -345,34 +351,45 @@ band_scan_kernel(uint4* __restrict__ rec, int tiles_per_worker, const uint32_t* 
     const int n = (int)tile_n[m];
     if (n == 0) return;
     uint4* r = rec + (int64_t)m * tiles_per_worker;
-    const int per = (n + kListThreads - 1) / kListThreads;
-    const int t0 = min((int)threadIdx.x * per, n), t1 = min(t0 + per, n);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int rows = (n + kListThreads - 1) / kListThreads;  // rows of 32 records per warp
+    const int t0 = warp * rows * 32;
     uint32_t sC = 0, sA = 0, sB = 0;
 #pragma unroll 4
-    for (int t = t0; t < t1; ++t) {
-        const uint4 x = r[t];
-        sC += x.x; sA += x.y; sB += x.z;
+    for (int i = 0; i < rows; ++i) {
+        const int t = t0 + i * 32 + lane;
+        if (t < n) {
+            const uint4 x = r[t];
+            sC += x.x; sA += x.y; sB += x.z;
+        }
     }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t iC = sC, iA = sA, iB = sB;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t yC = __shfl_up_sync(0xFFFFFFFFu, iC, o), yA = __shfl_up_sync(0xFFFFFFFFu, iA, o),
-                       yB = __shfl_up_sync(0xFFFFFFFFu, iB, o);
-        if (lane >= o) { iC += yC; iA += yA; iB += yB; }
-    }
-    if (lane == 31) { sh_w[0][warp] = iC; sh_w[1][warp] = iA; sh_w[2][warp] = iB; }
+    sC = __reduce_add_sync(0xFFFFFFFFu, sC);
+    sA = __reduce_add_sync(0xFFFFFFFFu, sA);
+    sB = __reduce_add_sync(0xFFFFFFFFu, sB);
+    if (lane == 0) { sh_w[0][warp] = sC; sh_w[1][warp] = sA; sh_w[2][warp] = sB; }
     __syncthreads();
-    uint32_t pC = iC - sC, pA = iA - sA, pB = iB - sB, totC = 0, totA = 0, totB = 0;
+    uint32_t pC = 0, pA = 0, pB = 0, totC = 0, totA = 0, totB = 0;  // running totals before this warp's range
     for (int w = 0; w < kListThreads / 32; ++w) {
         const uint32_t xC = sh_w[0][w], xA = sh_w[1][w], xB = sh_w[2][w];
         totC += xC; totA += xA; totB += xB;
         if (w < warp) { pC += xC; pA += xA; pB += xB; }
     }
-    for (int t = t0; t < t1; ++t) {
-        const uint4 x = r[t];
-        r[t] = make_uint4(pC, pA, pB, 0u);
-        pC += x.x; pA += x.y; pB += x.z;
+    for (int i = 0; i < rows; ++i) {
+        const int t = t0 + i * 32 + lane;
+        if (t0 + i * 32 >= n) break;  // warp-uniform
+        uint4 x = make_uint4(0u, 0u, 0u, 0u);
+        if (t < n) x = r[t];
+        uint32_t iC = x.x, iA = x.y, iB = x.z;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t yC = __shfl_up_sync(0xFFFFFFFFu, iC, o), yA = __shfl_up_sync(0xFFFFFFFFu, iA, o),
+                           yB = __shfl_up_sync(0xFFFFFFFFu, iB, o);
+            if (lane >= o) { iC += yC; iA += yA; iB += yB; }
+        }
+        if (t < n) r[t] = make_uint4(pC + iC - x.x, pA + iA - x.y, pB + iB - x.z, 0u);
+        pC += __shfl_sync(0xFFFFFFFFu, iC, 31);
+        pA += __shfl_sync(0xFFFFFFFFu, iA, 31);
+        pB += __shfl_sync(0xFFFFFFFFu, iB, 31);
     }
     if (threadIdx.x == 0) {
         const EmitParams e = emit[m];

@@ -275,6 +275,7 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand
     __shared__ uint32_t sh_tot[kResolveThreads], sh_off[kResolveThreads];
     __shared__ int sh_bin[kMaxQueries];
     __shared__ uint32_t sh_slot[kMaxQueries];
+    __shared__ bool sh_live[kMaxQueries];
     const int m = blockIdx.x;
     uint32_t* S = hist1 + (int64_t)m * kBins1;
     Query* q = queries + m * kMaxQueries;
@@ -321,35 +322,61 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand
     }
     __syncthreads();
     if (worker_err[m]) return;
-    if (threadIdx.x < nq && !q[threadIdx.x].trivial) {
-        Query& qq = q[threadIdx.x];
-        int lo = 0, hi = kBins1 - 1;  // largest b with S[b] >= k  (S[0] = d >= k)
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (S[mid] >= qq.k) lo = mid; else hi = mid - 1;
-        }
-        const uint32_t ab = (lo == kBins1 - 1) ? 0u : S[lo + 1];
-        if (is_bf16) {
-            qq.T = (uint32_t)lo;
-            qq.c = ab;
-            qq.n = S[lo] - ab;
-            qq.r = qq.k - ab;
-        } else {
-            qq.prefix = (uint32_t)lo << 16;
-            qq.rem = qq.k - ab;
+    {
+        // Warp j descends query j: the largest bin b with S[b] >= k (S[0] = d >= k).  S at the first bin of each of
+        // the 1024 groups of 32 bins is still in shared memory (group total + what lies above it), so two 32-way
+        // votes find the group and one coalesced row of S from memory finds the bin.
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        if (warp < nq && !q[warp].trivial) {
+            Query& qq = q[warp];
+            const uint32_t k = qq.k;
+            auto group_S = [&](int e) -> uint32_t { return sh_tot[e] + sh_off[e]; };
+            uint32_t mk = __ballot_sync(0xFFFFFFFFu, group_S(lane * 32) >= k);
+            const int coarse = 31 - __clz((int)mk);   // lane 0 always votes yes
+            mk = __ballot_sync(0xFFFFFFFFu, group_S(coarse * 32 + lane) >= k);
+            const int e = coarse * 32 + (31 - __clz((int)mk));
+            const uint32_t sb = S[e * 32 + lane];
+            mk = __ballot_sync(0xFFFFFFFFu, sb >= k);
+            const int in_group = 31 - __clz((int)mk);
+            const int lo = e * 32 + in_group;
+            const uint32_t next_in = __shfl_sync(0xFFFFFFFFu, sb, (in_group + 1) & 31);
+            const uint32_t s_lo = __shfl_sync(0xFFFFFFFFu, sb, in_group);
+            const uint32_t ab = (lo == kBins1 - 1) ? 0u : (in_group < 31 ? next_in : group_S(e + 1));
+            if (lane == 0) {
+                if (is_bf16) {
+                    qq.T = (uint32_t)lo;
+                    qq.c = ab;
+                    qq.n = s_lo - ab;
+                    qq.r = k - ab;
+                } else {
+                    qq.prefix = (uint32_t)lo << 16;
+                    qq.rem = k - ab;
+                }
+            }
         }
     }
     __syncthreads();
     if (is_bf16) return;
-    if (threadIdx.x == 0) assign_slots(q, nq, 16);
-    __syncthreads();
     if (threadIdx.x < nq) {
         const Query& qq = q[threadIdx.x];
         // trivial queries: "nothing inside" sits above every bin, "everything inside" below every bin
         sh_bin[threadIdx.x] = (qq.trivial == 2u) ? -1 : (qq.trivial ? kBins1 : (int)(qq.prefix >> 16));
-        sh_slot[threadIdx.x] = qq.slot;
+        sh_live[threadIdx.x] = qq.trivial == 0u;
     }
     __syncthreads();
+    if (threadIdx.x == 0) {  // slots of the second digit pass: live queries in the same bin share one
+        int next = 0;
+        for (int jq = 0; jq < nq; ++jq) {
+            sh_slot[jq] = kNoSlot;
+            if (!sh_live[jq]) continue;
+            int sl = -1;
+            for (int i = 0; i < jq; ++i)
+                if (sh_live[i] && sh_bin[i] == sh_bin[jq]) { sl = (int)sh_slot[i]; break; }
+            sh_slot[jq] = (sl >= 0) ? (uint32_t)sl : (uint32_t)next++;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < nq && sh_live[threadIdx.x]) q[threadIdx.x].slot = sh_slot[threadIdx.x];
     if (threadIdx.x == 0) {
         // the smallest key that can be a candidate: the lower edge of the lowest boundary bin (no live query: none)
         int lowest = kBins1;
@@ -379,16 +406,14 @@ resolve1_kernel(uint32_t* hist1, Query* queries, uint8_t* table1, uint32_t* cand
             atomicAdd(&bracket_stats[hit ? 0 : (had ? 1 : 2)], 1ull);
         }
     }
+    // code of bin b: the number of leading queries whose bin lies above b, or 64 + slot if the first one that does
+    // not lies in b itself.  That number can only grow as b falls, so the thread walks its bins downwards.
     uint8_t* tab = table1 + (int64_t)m * kBins1;
-    for (int i = 0; i < per; ++i) {
+    int j = 0;
+    for (int i = per - 1; i >= 0; --i) {
         const int b = i * kResolveThreads + threadIdx.x;
-        uint32_t code = 0;
-        for (int j = 0; j < nq; ++j) {
-            if (sh_bin[j] > b) ++code;
-            else if (sh_bin[j] == b) { code = 64u + sh_slot[j]; break; }
-            else break;  // bins are non-increasing in j
-        }
-        tab[b] = (uint8_t)code;
+        while (j < nq && sh_bin[j] > b) ++j;
+        tab[b] = (uint8_t)((j < nq && sh_bin[j] == b) ? 64u + sh_slot[j] : (uint32_t)j);
     }
 }
 
@@ -559,21 +584,21 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
 
 // Digit pass over the compacted candidate keys (normal case).
 template <int PASS>
-__global__ void __launch_bounds__(kSweepThreads)
-cand_pass_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const uint32_t* __restrict__ cand_count,
-                 const int* __restrict__ cand_overflow, const uint8_t* __restrict__ table1,
-                 const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err) {
-    __shared__ uint32_t sh_hist[kMaxQueries * kBins23];
+__device__ __forceinline__ void cand_pass_body(uint32_t* sh_hist, int bx, int nbx, const uint32_t* __restrict__ cand_keys,
+                                               int64_t cand_cap, const uint32_t* __restrict__ cand_count,
+                                               const int* __restrict__ cand_overflow, const uint8_t* __restrict__ table1,
+                                               const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out,
+                                               const int* worker_err) {
     const int m = blockIdx.y;
     if (worker_err[m] || cand_overflow[m]) return;
     const uint32_t n = cand_count[m];
-    if ((uint64_t)blockIdx.x * kSweepThreads >= n) return;
+    if ((uint64_t)bx * kSweepThreads >= n) return;
     for (int i = threadIdx.x; i < kMaxQueries * kBins23; i += blockDim.x) sh_hist[i] = 0;
     __syncthreads();
     const uint32_t* cand = cand_keys + (int64_t)m * cand_cap;
     const uint8_t* tab = table1 + (int64_t)m * kBins1;
     const uint8_t* mp = map2 + (int64_t)m * kMaxQueries * kBins23;
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    for (uint32_t i = bx * blockDim.x + threadIdx.x; i < n; i += nbx * blockDim.x) {
         const uint32_t key = cand[i];
         const uint32_t code = __ldg(&tab[key >> 16]);
         if (code < 64u) continue;  // a bracket bin that holds no threshold after all
@@ -654,11 +679,10 @@ cand_sums_kernel(const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const
 // large share of its entries falls into the boundary bins (many equal magnitudes)
 // -------------------------------------------------------------------------------------------
 template <int PASS>
-__global__ void __launch_bounds__(kSweepThreads)
-masked_pass_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uint8_t* __restrict__ table1,
-                   const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err,
-                   const int* __restrict__ cand_overflow) {
-    extern __shared__ uint8_t sh_raw[];
+__device__ __forceinline__ void masked_pass_body(uint8_t* sh_raw, int bx, int nbx, const float* __restrict__ g, int64_t d,
+                                                 int64_t ld, const uint8_t* __restrict__ table1,
+                                                 const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out,
+                                                 const int* worker_err, const int* __restrict__ cand_overflow) {
     uint32_t* sh_hist = reinterpret_cast<uint32_t*>(sh_raw);                        // [32][256]
     uint8_t* sh_table = sh_raw + kMaxQueries * kBins23 * sizeof(uint32_t);          // [32768]
     uint8_t* sh_map = sh_table + kBins1;                                            // [32][256] (pass 3)
@@ -678,7 +702,7 @@ masked_pass_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uin
     __syncthreads();
     const float* row = g + (int64_t)m * ld;
     int64_t v0, v1;
-    block_vector_range(d, 4, blockIdx.x, gridDim.x, &v0, &v1);
+    block_vector_range(d, 4, bx, nbx, &v0, &v1);
 #pragma unroll 4
     for (int64_t v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
         for_each_in_vector<float>(row, v, d, [&](int64_t, uint32_t bits) {
@@ -701,6 +725,23 @@ masked_pass_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const uin
         const uint32_t c = sh_hist[i];
         if (c) atomicAdd(&out[i], c);
     }
+}
+
+// One launch per digit pass: the first nb_cand blocks of a worker take its compacted candidate keys, the others are
+// the full-row fall-back (they return at once unless the worker's candidate buffer overflowed).
+template <int PASS>
+__global__ void __launch_bounds__(kSweepThreads)
+digit_pass_kernel(int nb_cand, const float* __restrict__ g, int64_t d, int64_t ld,
+                  const uint32_t* __restrict__ cand_keys, int64_t cand_cap, const uint32_t* __restrict__ cand_count,
+                  const int* __restrict__ cand_overflow, const uint8_t* __restrict__ table1,
+                  const uint8_t* __restrict__ map2, uint32_t* __restrict__ hist_out, const int* worker_err) {
+    extern __shared__ __align__(16) uint8_t sh_digit[];
+    if ((int)blockIdx.x < nb_cand)
+        cand_pass_body<PASS>(reinterpret_cast<uint32_t*>(sh_digit), blockIdx.x, nb_cand, cand_keys, cand_cap, cand_count,
+                             cand_overflow, table1, map2, hist_out, worker_err);
+    else
+        masked_pass_body<PASS>(sh_digit, blockIdx.x - nb_cand, gridDim.x - nb_cand, g, d, ld, table1, map2, hist_out,
+                               worker_err, cand_overflow);
 }
 
 // One warp per query walks its 256-bin histogram from the top digit down.
@@ -926,6 +967,8 @@ __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L,
                                   int64_t capacity, int* status, int* worker_err, int want_emit) {
     __shared__ double sh_delta[kMaxLevels];
     __shared__ double sh_p[kMaxLevels];
+    __shared__ uint32_t sh_T[kMaxQueries], sh_c[kMaxQueries], sh_n[kMaxQueries];
+    __shared__ bool sh_first[kMaxQueries];  // a live query whose threshold key no earlier live query has
     const int m = blockIdx.x;
     const Query* q = queries + m * kMaxQueries;
     if (worker_err[m]) {
@@ -933,6 +976,20 @@ __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L,
         return;
     }
     const int l = threadIdx.x;
+    if (adaptive) {
+        if (l < L - 1) {
+            sh_T[l] = q[l].trivial ? kKeyNone : q[l].T;
+            sh_c[l] = q[l].c;
+            sh_n[l] = q[l].n;
+        }
+        __syncwarp();
+        if (l < L - 1) {
+            bool first = !q[l].trivial;
+            for (int i = 0; i < l; ++i) first &= !(sh_T[i] == sh_T[l] && sh_T[i] != kKeyNone);
+            sh_first[l] = first;
+        }
+        __syncwarp();
+    }
     if (adaptive && l < L) {
         // open-interval energy: per-block partials added in block order (reproducible).
         // bf16 / overflowed fp32 worker: one source (histogram counts / full norm sweep);
@@ -956,14 +1013,11 @@ __global__ void probs_draw_kernel(const Query* queries, const int64_t* k, int L,
         }
         const int64_t lo = l ? k[l - 1] : 0, hi = k[l];
         for (int j = 0; j < L - 1; ++j) {
-            if (q[j].trivial) continue;
-            bool dup = false;
-            for (int i = 0; i < j; ++i) dup |= (!q[i].trivial && q[i].T == q[j].T);
-            if (dup) continue;
-            const int64_t c0 = q[j].c, c1 = c0 + (int64_t)q[j].n;
+            if (!sh_first[j]) continue;  // trivial, or the same threshold key as an earlier query
+            const int64_t c0 = sh_c[j], c1 = c0 + (int64_t)sh_n[j];
             const int64_t ov = min(c1, hi) - max(c0, lo);
             if (ov > 0) {
-                const uint32_t bits = is_bf16 ? (q[j].T << 16) : q[j].T;
+                const uint32_t bits = is_bf16 ? (sh_T[j] << 16) : sh_T[j];
                 const double x = (double)__uint_as_float(bits);
                 E = fma((double)ov, x * x, E);
             }
@@ -1205,27 +1259,15 @@ void launch_digit_pass(Workspace& ws, const void* g, int64_t d, int M, int64_t l
     const size_t smem = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
     const int nb_full = blocks_per_worker(ws, d, 4, kSweepThreads, M, 2);  // fall-back sweeps: a small grid, since they normally exit at once
     const int nb_cand = cand_blocks(ws, M);
-    if (pass == 2) {
-        {
-            LaunchScope t(ws, K_CAND2, s);
-            cand_pass_kernel<2><<<dim3(nb_cand, M), kSweepThreads, 0, s>>>(ws.cand_keys, ws.cand_cap, ws.cand_count,
-                                                                           ws.cand_overflow, ws.table1, ws.map2,
-                                                                           ws.hist2, ws.worker_err);
-        }
-        LaunchScope t(ws, K_MASKED2, s);
-        masked_pass_kernel<2><<<dim3(nb_full, M), kSweepThreads, smem, s>>>(
-            static_cast<const float*>(g), d, ld, ws.table1, ws.map2, ws.hist2, ws.worker_err, ws.cand_overflow);
-    } else {
-        {
-            LaunchScope t(ws, K_CAND3, s);
-            cand_pass_kernel<3><<<dim3(nb_cand, M), kSweepThreads, 0, s>>>(ws.cand_keys, ws.cand_cap, ws.cand_count,
-                                                                           ws.cand_overflow, ws.table1, ws.map2,
-                                                                           ws.hist3, ws.worker_err);
-        }
-        LaunchScope t(ws, K_MASKED3, s);
-        masked_pass_kernel<3><<<dim3(nb_full, M), kSweepThreads, smem, s>>>(
-            static_cast<const float*>(g), d, ld, ws.table1, ws.map2, ws.hist3, ws.worker_err, ws.cand_overflow);
-    }
+    LaunchScope t(ws, pass == 2 ? K_CAND2 : K_CAND3, s);
+    if (pass == 2)
+        digit_pass_kernel<2><<<dim3(nb_cand + nb_full, M), kSweepThreads, smem, s>>>(
+            nb_cand, static_cast<const float*>(g), d, ld, ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow,
+            ws.table1, ws.map2, ws.hist2, ws.worker_err);
+    else
+        digit_pass_kernel<3><<<dim3(nb_cand + nb_full, M), kSweepThreads, smem, s>>>(
+            nb_cand, static_cast<const float*>(g), d, ld, ws.cand_keys, ws.cand_cap, ws.cand_count, ws.cand_overflow,
+            ws.table1, ws.map2, ws.hist3, ws.worker_err);
 }
 
 void launch_resolve23(Workspace& ws, int M, int L, int pass, cudaStream_t s) {
@@ -1303,9 +1345,9 @@ int configure_select_kernels() {
                              (int)(kBins1 * sizeof(uint32_t)));
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     const int smem_masked = kMaxQueries * kBins23 * sizeof(uint32_t) + kBins1 + kMaxQueries * kBins23;
-    e = cudaFuncSetAttribute(masked_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_masked);
+    e = cudaFuncSetAttribute(digit_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_masked);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
-    e = cudaFuncSetAttribute(masked_pass_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_masked);
+    e = cudaFuncSetAttribute(digit_pass_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_masked);
     if (e != cudaSuccess) return MLMC_ERR_CUDA;
     e = cudaFuncSetAttribute(norm_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxLevels * kSweepThreads * sizeof(double)));
