@@ -174,15 +174,15 @@ __device__ __forceinline__ uint32_t batch_flags(const uint32_t (&w)[kEmitRows], 
 // The same flags for the write pass, with the ties as masks instead of counts: bit i (fp32) or bits i and 16 + i
 // (bf16 low / high half) of mA / mB = word i of this lane holds a key equal to Ta / Tb.
 template <typename T>
-__device__ __forceinline__ uint32_t batch_masks(const uint32_t (&w)[kEmitRows], uint32_t Tb, uint32_t Ta, uint32_t* mA,
-                                                uint32_t* mB) {
-    uint32_t flags = 0, a = 0, b = 0;
+__device__ __forceinline__ uint32_t batch_masks(const uint32_t (&w)[kEmitRows], uint32_t Tb, uint32_t Ta, bool ties,
+                                                uint32_t* mA, uint32_t* mB) {
+    uint32_t flags = 0, a = 0, b = 0;  // ties = false: the tile holds no key equal to a threshold, the masks stay empty
     if constexpr (EmitWord<T>::S == 1) {
         const uint32_t W = Ta - Tb;
 #pragma unroll
         for (int i = 0; i < kEmitRows; ++i)
             if (((w[i] & 0x7FFFFFFFu) - Tb) <= W) flags |= 1u << i;
-        if (__any_sync(0xFFFFFFFFu, flags != 0u)) {
+        if (ties && __any_sync(0xFFFFFFFFu, flags != 0u)) {
 #pragma unroll
             for (int i = 0; i < kEmitRows; ++i) {
                 const uint32_t tk = (w[i] & 0x7FFFFFFFu) - Tb;
@@ -200,7 +200,7 @@ __device__ __forceinline__ uint32_t batch_masks(const uint32_t (&w)[kEmitRows], 
             const uint32_t k2 = w[i] & 0x7FFF7FFFu;
             flags |= ((k2 + geB) & (leA - k2) & hi) >> (15 - i);
         }
-        if (__any_sync(0xFFFFFFFFu, flags != 0u)) {
+        if (ties && __any_sync(0xFFFFFFFFu, flags != 0u)) {
 #pragma unroll
             for (int i = 0; i < kEmitRows; ++i) {
                 const uint32_t k2 = w[i] & 0x7FFF7FFFu;
@@ -335,7 +335,9 @@ band_count_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
         }
         const uint32_t totCA = __reduce_add_sync(0xFFFFFFFFu, cC | (cA << 16));  // at most 8192 elements per tile
         cB = __reduce_add_sync(0xFFFFFFFFu, cB);
-        if (lane == 0) rec[(int64_t)m * tiles_per_worker + j] = make_uint4(totCA & 0xFFFFu, totCA >> 16, cB, 0u);
+        // the fourth word tells the write pass whether the tile holds a key equal to a threshold at all
+        if (lane == 0)
+            rec[(int64_t)m * tiles_per_worker + j] = make_uint4(totCA & 0xFFFFu, totCA >> 16, cB, ((totCA >> 16) | cB) ? 1u : 0u);
     }
 }
 
@@ -386,7 +388,7 @@ band_scan_kernel(uint4* __restrict__ rec, int tiles_per_worker, const uint32_t* 
                            yB = __shfl_up_sync(0xFFFFFFFFu, iB, o);
             if (lane >= o) { iC += yC; iA += yA; iB += yB; }
         }
-        if (t < n) r[t] = make_uint4(pC + iC - x.x, pA + iA - x.y, pB + iB - x.z, 0u);
+        if (t < n) r[t] = make_uint4(pC + iC - x.x, pA + iA - x.y, pB + iB - x.z, x.w);
         pC += __shfl_sync(0xFFFFFFFFu, iC, 31);
         pA += __shfl_sync(0xFFFFFFFFu, iA, 31);
         pB += __shfl_sync(0xFFFFFFFFu, iB, 31);
@@ -434,6 +436,7 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
         float* val_w = val_out + (int64_t)m * capacity;
         const uint4 pre = __ldg(&rec[(int64_t)m * tiles_per_worker + j]);
         uint32_t rC = pre.x, rA = pre.y, rB = pre.z;  // running totals before the current batch
+        const bool tile_ties = pre.w != 0u;           // found by the count pass
         __syncwarp();  // the previous tile's last batches have been read by every lane
         copy_batch_async<T>(row, d, tile, 0, lane, ring);
         cp_async_commit();
@@ -454,7 +457,7 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
                 cur[4 * q + 0] = x.x; cur[4 * q + 1] = x.y; cur[4 * q + 2] = x.z; cur[4 * q + 3] = x.w;
             }
             uint32_t mA, mB;
-            uint32_t member = batch_masks<T>(cur, Tb, Ta, &mA, &mB);
+            uint32_t member = batch_masks<T>(cur, Tb, Ta, tile_ties, &mA, &mB);
             if (!__any_sync(0xFFFFFFFFu, member != 0u)) continue;  // no closed-range key in the batch: nothing to count either
             const uint32_t nC = __popc(member), nA = __popc(mA), nB = __popc(mB);
             const uint32_t totCA = __reduce_add_sync(0xFFFFFFFFu, nC | (nA << 16));
