@@ -37,7 +37,9 @@ __device__ __forceinline__ RtnGrid rtn_grid(float c, int r) {
 
 __device__ __forceinline__ float rtn_value(float v, float c, RtnGrid gq) {
     const float t = __fmul_rn(v, gq.inv);
-    const float k = rintf(t);  // to nearest, ties to even
+    // to nearest, ties to even: |t| <= 2^15 (r <= 16), so adding and subtracting 1.5 * 2^23 rounds t to an integer in
+    // the adder, with the default rounding mode, without the conversion unit
+    const float k = __fadd_rn(__fadd_rn(t, 12582912.0f), -12582912.0f);
     return fminf(fmaxf(__fmul_rn(k, gq.delta), -c), c);
 }
 
