@@ -30,11 +30,12 @@ int mlmc_timing_read(mlmc_ctx* ctx, double* total_ms, int64_t* launches, void* s
  * copied to u_host[M].  Synchronous; for checking the counter generator against known answers. */
 int mlmc_read_u(mlmc_ctx* ctx, uint64_t seed, uint64_t step, int M, double* u_host, void* stream);
 
-/* How much of every row the last mlmc_compress_topk on this context read when it emitted the bands (the
- * band of ranks (k_{l-1}, k_l] of Sec. 3.2): the emission reads only the tiles of 4096 32-bit words (4096 fp32
- * or 8192 bf16 entries) whose largest magnitude reaches the band's lower threshold, twice each.
- *   listed_host  host uint32 [M]: tiles of worker m that were read.
- *   tiles_host   host int64: tiles in one row.
+/* How much of every row the last mlmc_compress_topk / mlmc_compress_stopk on this context read when it emitted the
+ * bands (the band of ranks (k_{l-1}, k_l] of Sec. 3.2): the emission reads only the batches of 512 32-bit words
+ * (512 fp32 or 1024 bf16 entries; eight batches make a tile) whose largest magnitude reaches the band's lower
+ * threshold, twice each.
+ *   listed_host  host uint32 [M]: batches of worker m that were read.
+ *   tiles_host   host int64: batches in one row (the ragged last tile counted whole).
  * Synchronous (copies from the device and waits for the stream); a measurement aid, not part of the method. */
 int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t* tiles_host, void* stream);
 

@@ -204,7 +204,8 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_u = pl.take(sizeof(double) * M_max);
     const size_t o_emit = pl.take(sizeof(EmitParams) * M_max);
     const size_t o_tdesc = pl.take(sizeof(uint4) * ws.max_tiles);
-    const size_t o_tmax = pl.take(sizeof(uint32_t) * ws.max_tiles);
+    const size_t o_tmax = pl.take(sizeof(uint32_t) * ws.max_tiles * kEmitGroups);
+    const size_t o_groupn = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_wtiles = pl.take(sizeof(uint32_t) * ws.max_tiles);
     const size_t o_tilen = pl.take(sizeof(uint32_t) * M_max);
     const size_t o_cfloor = pl.take(sizeof(uint32_t) * M_max);
@@ -261,6 +262,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     ws.tile_max = reinterpret_cast<uint32_t*>(base + o_tmax);
     ws.worker_tiles = reinterpret_cast<uint32_t*>(base + o_wtiles);
     ws.tile_n = reinterpret_cast<uint32_t*>(base + o_tilen);
+    ws.group_n = reinterpret_cast<uint32_t*>(base + o_groupn);
     ws.cand_floor = reinterpret_cast<uint32_t*>(base + o_cfloor);
     ws.agg_offsets = reinterpret_cast<uint32_t*>(base + o_aggoff);
     ws.gmax_bits = reinterpret_cast<uint32_t*>(base + o_gmax);
@@ -387,8 +389,8 @@ int mlmc_read_listed_tiles(mlmc_ctx* ctx, int M, uint32_t* listed_host, int64_t*
     if (!ctx || !listed_host || !tiles_host || M < 1 || M > ctx->ws.M_max) return MLMC_ERR_ARG;
     DeviceGuard guard(ctx->ws.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    *tiles_host = ctx->ws.last_emit_tiles;
-    if (cudaMemcpyAsync(listed_host, ctx->ws.tile_n, sizeof(uint32_t) * M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    *tiles_host = ctx->ws.last_emit_tiles * kEmitGroups;
+    if (cudaMemcpyAsync(listed_host, ctx->ws.group_n, sizeof(uint32_t) * M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return MLMC_ERR_CUDA;
     return finish(cudaStreamSynchronize(s));
 }

@@ -21,6 +21,8 @@ constexpr int kEmitMaxWorkers = 1024;         // M of one call: the emit and ave
 constexpr int kEmitRows = 16;                 // 32-bit words per lane that a warp of the emit kernels holds at a time
 constexpr int kEmitTile = 4096;               // 32-bit words per emit tile (1 fp32 or 2 bf16 elements each); one warp per tile
 constexpr int kEmitTileVecs = kEmitTile / 4;  // 16-byte vectors per tile, for both element types
+constexpr int kEmitGroups = kEmitTile / (kEmitRows * 32);  // batches of kEmitRows * 32 words per tile: 8
+constexpr int kEmitGroupVecs = kEmitTileVecs / kEmitGroups;  // 16-byte vectors per batch: 128
 constexpr int kAggTile = 4096;                // dense output elements per aggregation tile
 
 // Per-worker selection query: the rank-k element of the total order.
@@ -97,9 +99,10 @@ struct Workspace {
     EmitParams* emit;            // [M]
     uint4* tile_desc;            // [M][tiles per worker] per listed tile {C, A, B}: its own counts, then the running totals before it
     int64_t max_tiles;
-    uint32_t* tile_max;          // [M][tiles per worker] largest magnitude key of every emit tile (sweep 1)
-    uint32_t* worker_tiles;      // [M][tiles per worker] the tiles of a worker that can hold band entries, ascending
+    uint32_t* tile_max;          // [M][tiles per worker][kEmitGroups] largest magnitude key of every batch of every emit tile (sweep 1)
+    uint32_t* worker_tiles;      // [M][tiles per worker] the tiles of a worker that can hold band entries, ascending: tile | batch mask << 24
     uint32_t* tile_n;            // [M] how many of them
+    uint32_t* group_n;           // [M] how many batches they have to read
     int64_t last_emit_tiles;     // tiles per row of the last emission (host side, for mlmc_read_listed_tiles)
     uint32_t* cand_floor;        // [M] smallest key that can be a candidate of sweep 2 (lower edge of the lowest boundary bin)
     uint32_t* agg_offsets;       // [M][agg_tiles_max + 1]

@@ -255,32 +255,45 @@ constexpr int kListThreads = 1024;
 
 __global__ void __launch_bounds__(kListThreads)
 tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, const EmitParams* __restrict__ emit,
-                 uint32_t key_cap, uint32_t* __restrict__ worker_tiles, uint32_t* __restrict__ tile_n, int* status) {
-    __shared__ uint32_t sh_warp[kListThreads / 32];
+                 uint32_t key_cap, uint32_t* __restrict__ worker_tiles, uint32_t* __restrict__ tile_n,
+                 uint32_t* __restrict__ group_n, int* status) {
+    __shared__ uint32_t sh_warp[kListThreads / 32], sh_grp[kListThreads / 32];
     const int m = blockIdx.x;
     const EmitParams e = emit[m];
     const bool on = e.enabled && e.level >= 0 && e.expect > 0u;
     const uint32_t Tb = min(e.Tb, key_cap);
-    const uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker;
+    // the batch maxima of a tile are two 16-byte vectors; a batch below Tb holds no band entry and no tie of Tb
+    const uint4* tmax = reinterpret_cast<const uint4*>(tile_max + (int64_t)m * tiles_per_worker * kEmitGroups);
     uint32_t* list = worker_tiles + (int64_t)m * tiles_per_worker;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rows = (tiles_per_worker + kListThreads - 1) / kListThreads;  // rows of 32 tiles per warp
     const int t0 = warp * rows * 32;
-    uint32_t mine = 0;  // listed tiles of this warp (the same in every lane)
+    auto batch_mask = [&](int t) -> uint32_t {
+        if (t >= tiles_per_worker) return 0u;
+        const uint4 a = __ldg(&tmax[2 * (int64_t)t]), b = __ldg(&tmax[2 * (int64_t)t + 1]);
+        return (a.x >= Tb ? 1u : 0u) | (a.y >= Tb ? 2u : 0u) | (a.z >= Tb ? 4u : 0u) | (a.w >= Tb ? 8u : 0u) |
+               (b.x >= Tb ? 16u : 0u) | (b.y >= Tb ? 32u : 0u) | (b.z >= Tb ? 64u : 0u) | (b.w >= Tb ? 128u : 0u);
+    };
+    uint32_t mine = 0, groups = 0;  // listed tiles of this warp (the same in every lane), batches of this lane
     if (on) {
 #pragma unroll 4
         for (int r = 0; r < rows; ++r) {
-            const int t = t0 + r * 32 + lane;
-            const bool f = t < tiles_per_worker && __ldg(&tmax[t]) >= Tb;
-            mine += __popc(__ballot_sync(0xFFFFFFFFu, f));
+            const uint32_t bm = batch_mask(t0 + r * 32 + lane);
+            mine += __popc(__ballot_sync(0xFFFFFFFFu, bm != 0u));
+            groups += __popc(bm);
         }
     }
-    if (lane == 0) sh_warp[warp] = mine;
+    groups = __reduce_add_sync(0xFFFFFFFFu, groups);
+    if (lane == 0) {
+        sh_warp[warp] = mine;
+        sh_grp[warp] = groups;
+    }
     __syncthreads();
-    uint32_t before = 0, total = 0;
+    uint32_t before = 0, total = 0, total_groups = 0;
     for (int w = 0; w < kListThreads / 32; ++w) {
         const uint32_t x = sh_warp[w];
         total += x;
+        total_groups += sh_grp[w];
         if (w < warp) before += x;
     }
     if (on && mine) {
@@ -289,14 +302,15 @@ tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, co
 #pragma unroll 4
         for (int r = 0; r < rows; ++r) {
             const int t = t0 + r * 32 + lane;
-            const bool f = t < tiles_per_worker && __ldg(&tmax[t]) >= Tb;
-            const uint32_t mk = __ballot_sync(0xFFFFFFFFu, f);
-            if (f) list[pos + __popc(mk & lt)] = (uint32_t)t;
+            const uint32_t bm = batch_mask(t);
+            const uint32_t mk = __ballot_sync(0xFFFFFFFFu, bm != 0u);
+            if (bm) list[pos + __popc(mk & lt)] = (uint32_t)t | (bm << 24);  // tile numbers stay below 2^20
             pos += __popc(mk);
         }
     }
     if (threadIdx.x == 0) {
         tile_n[m] = total;
+        group_n[m] = total_groups;
         if (on && total == 0u) set_status(status, MLMC_ERR_INTERNAL);  // a band with entries lies in some tile
     }
 }
@@ -316,15 +330,22 @@ band_count_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
     for (uint32_t f = blockIdx.x * (kBandThreads / 32) + (threadIdx.x >> 5); f < total; f += warps) {
         const int m = worker_of(sh_off, M, f);
         const uint32_t j = f - sh_off[m];
-        const int64_t tile = worker_tiles[(int64_t)m * tiles_per_worker + j];
+        const uint32_t entry = worker_tiles[(int64_t)m * tiles_per_worker + j];
+        const int64_t tile = entry & 0xFFFFFFu;
+        uint32_t todo = entry >> 24;  // the batches of the tile that can hold band entries (at least one)
         const uint32_t Tb = min(__ldg(&emit[m].Tb), EW::kCap), Ta = min(__ldg(&emit[m].Ta), EW::kCap);
         const T* row = g + (int64_t)m * ld;
         uint32_t cC = 0, cA = 0, cB = 0;
         uint32_t cur[kEmitRows], nxt[kEmitRows];
-        load_batch<T>(row, d, tile, 0, lane, cur);
+        load_batch<T>(row, d, tile, __ffs(todo) - 1, lane, cur);
+        todo &= todo - 1u;
 #pragma unroll 1
-        for (int b = 0; b < kBatches; ++b) {
-            if (b + 1 < kBatches) load_batch<T>(row, d, tile, b + 1, lane, nxt);  // in flight while this batch is counted
+        for (bool more = true; more;) {
+            more = todo != 0u;
+            if (more) {  // in flight while this batch is counted
+                load_batch<T>(row, d, tile, __ffs(todo) - 1, lane, nxt);
+                todo &= todo - 1u;
+            }
             uint32_t a1, b1;
             const uint32_t flags = batch_flags<T>(cur, Tb, Ta, &a1, &b1);
             cC += __popc(flags);
@@ -426,7 +447,8 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
     for (uint32_t f = blockIdx.x * (kBandThreads / 32) + (threadIdx.x >> 5); f < total; f += warps) {
         const int m = worker_of(sh_off, M, f);
         const uint32_t j = f - sh_off[m];
-        const int64_t tile = worker_tiles[(int64_t)m * tiles_per_worker + j];
+        const uint32_t entry = worker_tiles[(int64_t)m * tiles_per_worker + j];
+        const int64_t tile = entry & 0xFFFFFFu;
         const EmitParams ep = emit[m];
         const uint32_t Tb = min(ep.Tb, EW::kCap), Ta = min(ep.Ta, EW::kCap);
         const uint32_t W = Ta - Tb;
@@ -437,19 +459,31 @@ band_write_kernel(const T* __restrict__ g, int64_t d, int64_t ld, int tiles_per_
         const uint4 pre = __ldg(&rec[(int64_t)m * tiles_per_worker + j]);
         uint32_t rC = pre.x, rA = pre.y, rB = pre.z;  // running totals before the current batch
         const bool tile_ties = pre.w != 0u;           // found by the count pass
+        // Only the batches of the tile that can hold band entries are read (mask from the listing): `todo` walks them
+        // for processing, `ahead` two batches further for the copies.
+        uint32_t todo = entry >> 24, ahead = todo;
         __syncwarp();  // the previous tile's last batches have been read by every lane
-        copy_batch_async<T>(row, d, tile, 0, lane, ring);
+        copy_batch_async<T>(row, d, tile, __ffs(ahead) - 1, lane, ring);
+        ahead &= ahead - 1u;
         cp_async_commit();
-        copy_batch_async<T>(row, d, tile, 1, lane, ring + kBatchWords);
+        if (ahead) {
+            copy_batch_async<T>(row, d, tile, __ffs(ahead) - 1, lane, ring + kBatchWords);
+            ahead &= ahead - 1u;
+        }
         cp_async_commit();
 #pragma unroll 1
-        for (int b = 0; b < kBatches; ++b) {
-            __syncwarp();  // batch b - 1 has been read by every lane: its slot takes batch b + 2
-            if (b + 2 < kBatches) copy_batch_async<T>(row, d, tile, b + 2, lane, ring + ((b + 2) % kWriteSlots) * kBatchWords);
+        for (int it = 0; todo; ++it) {
+            const int b = __ffs(todo) - 1;
+            todo &= todo - 1u;
+            __syncwarp();  // the batch before this one has been read by every lane: its slot takes the copy two ahead
+            if (ahead) {
+                copy_batch_async<T>(row, d, tile, __ffs(ahead) - 1, lane, ring + ((it + 2) % kWriteSlots) * kBatchWords);
+                ahead &= ahead - 1u;
+            }
             cp_async_commit();  // one group per step, empty at the end of the tile
-            cp_async_wait<2>();  // batch b has landed
+            cp_async_wait<2>();  // this batch has landed
             __syncwarp();
-            const uint32_t* slot = ring + (b % kWriteSlots) * kBatchWords;
+            const uint32_t* slot = ring + (it % kWriteSlots) * kBatchWords;
             uint32_t cur[kEmitRows];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -683,7 +717,7 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
     {
         LaunchScope t(ws, K_TILE_LIST, s);
         tile_list_kernel<<<M, kListThreads, 0, s>>>(ws.tile_max, tpw, ws.emit, dtype == MLMC_BF16 ? 0x7F80u : 0x7F800000u,
-                                                    ws.worker_tiles, ws.tile_n, ws.status);
+                                                    ws.worker_tiles, ws.tile_n, ws.group_n, ws.status);
     }
     const int wpb = kBandThreads / 32;
     const size_t smem = (size_t)(M + 1) * sizeof(uint32_t);

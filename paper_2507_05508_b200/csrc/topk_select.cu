@@ -90,9 +90,9 @@ __global__ void uniforms_kernel(double* u_dev, int M, uint64_t seed, uint64_t st
 // -------------------------------------------------------------------------------------------
 // sweep 1: leading-digit histogram of every worker (shared-memory counts, flushed with atomics)
 // -------------------------------------------------------------------------------------------
-// The sweep also records the largest key of every emit tile (kEmitTileVecs consecutive 16-byte vectors of the
-// row): the emit sweep reads only the tiles whose largest key reaches the lower threshold of the drawn band.
-// Chunks start at a multiple of 32 vectors, so the 32 vectors a warp loads together lie in one tile.
+// The sweep also records the largest key of every batch of the emit tiles (kEmitGroupVecs consecutive 16-byte
+// vectors of the row): the emit sweep reads only the batches whose largest key reaches the lower threshold of the
+// drawn band.  Chunks start at a multiple of 32 vectors, so the 32 vectors a warp loads together lie in one batch.
 // BR (fp32, fixed p): the keys whose leading digit lies in one of the worker's two brackets (the bins around last
 // call's boundary bins) are collected as candidates in the same sweep.  Every warp stages them in a private
 // shared-memory buffer, in lane order by a warp scan, and moves the buffer to the candidate list when it fills up
@@ -142,7 +142,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
     for (int b = threadIdx.x; b < kBins1; b += blockDim.x) sh_hist[b] = 0;
     __syncthreads();
     const T* row = g + (int64_t)m * ld;
-    uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker;
+    uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker * kEmitGroups;  // one slot per batch of kEmitGroupVecs vectors
     const int64_t nvec = (d + Tr::kVec - 1) / Tr::kVec;
     bool bad = false;
     auto count_key = [&](uint32_t bits) { atomicAdd(&sh_hist[Tr::key(bits) >> Tr::kShift1], 1u); };  // Inf / NaN: see the maxima
@@ -177,7 +177,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
                     }
                 });
                 bad |= vm >= Tr::kInfKey;
-                atomicMax(&tmax[u / kEmitTileVecs], vm);
+                atomicMax(&tmax[u / kEmitGroupVecs], vm);
             }
             break;
         }
@@ -194,7 +194,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
             }
             const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, vector_max(q[j]));
             bad |= wm >= Tr::kInfKey;  // a non-finite entry shows in the largest key of its warp
-            if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitTileVecs], wm);
+            if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitGroupVecs], wm);
         }
         if constexpr (BR) {
             uint32_t cm = 0;  // bit 4 j + e: element e of vector j lies in a bracket
@@ -473,10 +473,13 @@ sums_candidates_kernel(const float* __restrict__ g, int64_t d, int64_t ld, const
     __shared__ uint8_t sh_want[kWantFlags];
     if (!SUMS) {
         const uint32_t floor_key = cand_floor[m];
-        const uint32_t* tmax = tile_max + (int64_t)m * tiles_per_worker + blockIdx.x;
+        const uint4* tmax = reinterpret_cast<const uint4*>(tile_max + ((int64_t)m * tiles_per_worker + blockIdx.x) * kEmitGroups);
         const int64_t nrounds = (v1 - v0 + vstep - 1) / vstep;
-        for (int r = threadIdx.x; r < kWantFlags && r < nrounds; r += kS2Threads)
-            sh_want[r] = tmax[(int64_t)r * gridDim.x] >= floor_key;
+        static_assert(kEmitGroups == 8, "a tile's batch maxima are two 16-byte vectors");
+        for (int r = threadIdx.x; r < kWantFlags && r < nrounds; r += kS2Threads) {
+            const uint4 a = tmax[(int64_t)r * gridDim.x * 2], b = tmax[(int64_t)r * gridDim.x * 2 + 1];
+            sh_want[r] = max(max(max(a.x, a.y), max(a.z, a.w)), max(max(b.x, b.y), max(b.z, b.w))) >= floor_key;
+        }
         __syncthreads();
     }
     auto wanted = [&](int64_t vb) -> bool {  // block-uniform
@@ -1182,7 +1185,7 @@ void launch_reset_selection(Workspace& ws, int dtype, int64_t d, int M, cudaStre
         ++r.n;
     };
     add(ws.hist1, (size_t)M * kBins1 * sizeof(uint32_t), 0u);
-    add(ws.tile_max, (size_t)M * tpw * sizeof(uint32_t), 0u);
+    add(ws.tile_max, (size_t)M * tpw * kEmitGroups * sizeof(uint32_t), 0u);
     if (dtype == MLMC_F32) {
         add(ws.cand_count, sizeof(uint32_t) * M, 0u);
         add(ws.cand_overflow, sizeof(int) * M, 0u);

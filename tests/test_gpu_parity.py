@@ -282,12 +282,13 @@ def test_topk_single_level_is_identity(B, ora, ctx):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_emission_reads_only_tiles_that_can_hold_band_entries(B, ctx, dtype):
-    """The emission lists, per worker, the tiles (4096 32-bit words) whose largest magnitude reaches the band's lower
-    threshold.  The list must cover every tile that holds a band entry, stay within the row, and be the whole row
-    for the last level (whose lower threshold is zero); a gradient with one loud layer lists few tiles."""
+def test_emission_reads_only_batches_that_can_hold_band_entries(B, ctx, dtype):
+    """The emission lists, per worker, the batches (512 32-bit words; eight per tile) whose largest magnitude reaches
+    the band's lower threshold.  The list must cover every batch that holds a band entry, stay within the row, and be
+    the whole row for the last level (whose lower threshold is zero); a gradient with one loud layer lists few."""
     per_word = 2 if dtype == "bf16" else 1
-    tile = 4096 * per_word
+    batch = 512 * per_word
+    tile = 8 * batch
     M, d = 4, 40 * tile + 123
     rng = np.random.default_rng(5)
     g_np = (rng.standard_normal((M, d)) * 1e-3).astype(np.float32)
@@ -297,20 +298,20 @@ def test_emission_reads_only_tiles_that_can_hold_band_entries(B, ctx, dtype):
         g = padded(g.to(torch.bfloat16), 8)
     k = [64, 1024, d]
     out = B.TopkBuffers(M, d)
-    tiles_in_row = (d + tile - 1) // tile
+    batches_in_row = (d + tile - 1) // tile * 8
     for step, p in ((0, [0.98, 0.01, 0.01]), (1, [0.01, 0.98, 0.01]), (2, [0.005, 0.005, 0.99])):
         B.mlmc_compress_topk(ctx, g, k, p, 11, step, out)
         assert B.mlmc_get_status(ctx) == B.MLMC_OK
-        listed, tiles = B.mlmc_read_listed_tiles(ctx, M)
-        assert tiles == tiles_in_row
+        listed, batches = B.mlmc_read_listed_tiles(ctx, M)
+        assert batches == batches_in_row
         for m in range(M):
             n, lv = int(out.count[m]), int(out.level[m])
-            touched = torch.unique((out.idx[m, :n].to(torch.int64) & 0xFFFFFFFF) // tile).numel()
-            assert touched <= listed[m] <= tiles
+            touched = torch.unique((out.idx[m, :n].to(torch.int64) & 0xFFFFFFFF) // batch).numel()
+            assert touched <= listed[m] <= batches
             if lv == 2:
-                assert listed[m] == tiles                   # everything below k_1: every tile can hold entries
+                assert listed[m] == batches                 # everything below k_1: every batch can hold entries
             else:
-                assert listed[m] <= 4                       # the loud layer (two tiles, at most one more on each side)
+                assert listed[m] <= 16                      # only batches of the loud layer (two tiles)
 
 
 def test_many_workers_and_the_maximum_number_of_levels(B, ora):
