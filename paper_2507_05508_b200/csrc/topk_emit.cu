@@ -256,8 +256,9 @@ constexpr int kListThreads = 1024;
 __global__ void __launch_bounds__(kListThreads)
 tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, const EmitParams* __restrict__ emit,
                  uint32_t key_cap, uint32_t* __restrict__ worker_tiles, uint32_t* __restrict__ tile_n,
-                 uint32_t* __restrict__ group_n, int* status) {
+                 uint32_t* __restrict__ group_n, int* status, int cached) {
     __shared__ uint32_t sh_warp[kListThreads / 32], sh_grp[kListThreads / 32];
+    extern __shared__ uint8_t sh_mask[];  // [tiles_per_worker] batch masks of the counting pass, when they fit (cached != 0)
     const int m = blockIdx.x;
     const EmitParams e = emit[m];
     const bool on = e.enabled && e.level >= 0 && e.expect > 0u;
@@ -278,7 +279,9 @@ tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, co
     if (on) {
 #pragma unroll 4
         for (int r = 0; r < rows; ++r) {
-            const uint32_t bm = batch_mask(t0 + r * 32 + lane);
+            const int t = t0 + r * 32 + lane;
+            const uint32_t bm = batch_mask(t);
+            if (cached && t < tiles_per_worker) sh_mask[t] = (uint8_t)bm;  // read back by this same thread below
             mine += __popc(__ballot_sync(0xFFFFFFFFu, bm != 0u));
             groups += __popc(bm);
         }
@@ -302,7 +305,7 @@ tile_list_kernel(const uint32_t* __restrict__ tile_max, int tiles_per_worker, co
 #pragma unroll 4
         for (int r = 0; r < rows; ++r) {
             const int t = t0 + r * 32 + lane;
-            const uint32_t bm = batch_mask(t);
+            const uint32_t bm = cached ? (t < tiles_per_worker ? (uint32_t)sh_mask[t] : 0u) : batch_mask(t);
             const uint32_t mk = __ballot_sync(0xFFFFFFFFu, bm != 0u);
             if (bm) list[pos + __popc(mk & lt)] = (uint32_t)t | (bm << 24);  // tile numbers stay below 2^20
             pos += __popc(mk);
@@ -703,7 +706,8 @@ aggregate_topk_warps_kernel(const uint32_t* __restrict__ idx, const float* __res
 int configure_emit_kernels() {  // the write pass: 48 KB ring + the list offsets of up to kEmitMaxWorkers workers
     const int smem = (kBandThreads / 32) * kWriteSlots * kBatchWords * (int)sizeof(uint32_t) +
                      (kEmitMaxWorkers + 1) * (int)sizeof(uint32_t);
-    if (cudaFuncSetAttribute(band_write_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+    if (cudaFuncSetAttribute(tile_list_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(band_write_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
         cudaFuncSetAttribute(band_write_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return MLMC_ERR_CUDA;
     return MLMC_OK;
@@ -716,8 +720,10 @@ void launch_emit(Workspace& ws, const void* g, int dtype, int64_t d, int M, int6
     ws.last_emit_tiles = tpw;
     {
         LaunchScope t(ws, K_TILE_LIST, s);
-        tile_list_kernel<<<M, kListThreads, 0, s>>>(ws.tile_max, tpw, ws.emit, dtype == MLMC_BF16 ? 0x7F80u : 0x7F800000u,
-                                                    ws.worker_tiles, ws.tile_n, ws.group_n, ws.status);
+        const int cached = tpw <= 96 * 1024;  // one byte per tile in shared memory
+        tile_list_kernel<<<M, kListThreads, cached ? (size_t)tpw : 0, s>>>(
+            ws.tile_max, tpw, ws.emit, dtype == MLMC_BF16 ? 0x7F80u : 0x7F800000u, ws.worker_tiles, ws.tile_n, ws.group_n,
+            ws.status, cached);
     }
     const int wpb = kBandThreads / 32;
     const size_t smem = (size_t)(M + 1) * sizeof(uint32_t);

@@ -118,6 +118,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
         if (br.z != 0xFFFFFFFFu) { lo_b = br.z << 16; span_b = ((br.w + 1u) << 16) - 1u; }
         if ((threadIdx.x & 31) == 0) *wcount = 0u;
     }
+    const uint32_t lo_min = min(lo_a, lo_b);
     auto in_bracket = [&](uint32_t bits) -> bool {
         const uint32_t key = bits & 0x7FFFFFFFu;
         return (key - lo_a) <= span_a || (key - lo_b) <= span_b;  // an empty bracket: key - lo wraps to key + 1 > 0
@@ -182,6 +183,7 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
             break;
         }
         uint4 q[kBatch];
+        uint32_t vmax[kBatch];  // BR only
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) q[j] = __ldg(reinterpret_cast<const uint4*>(row) + v + (int64_t)j * blockDim.x);
 #pragma unroll
@@ -192,7 +194,9 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
                 count_key(q[j].x & 0xFFFFu); count_key(q[j].x >> 16); count_key(q[j].y & 0xFFFFu); count_key(q[j].y >> 16);
                 count_key(q[j].z & 0xFFFFu); count_key(q[j].z >> 16); count_key(q[j].w & 0xFFFFu); count_key(q[j].w >> 16);
             }
-            const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, vector_max(q[j]));
+            const uint32_t vm = vector_max(q[j]);
+            if (BR) vmax[j] = vm;
+            const uint32_t wm = __reduce_max_sync(0xFFFFFFFFu, vm);
             bad |= wm >= Tr::kInfKey;  // a non-finite entry shows in the largest key of its warp
             if (lane == 0) atomicMax(&tmax[(v + (int64_t)j * blockDim.x) / kEmitGroupVecs], wm);
         }
@@ -200,10 +204,12 @@ hist1_kernel(const T* __restrict__ g, int64_t d, int64_t ld, uint32_t* __restric
             uint32_t cm = 0;  // bit 4 j + e: element e of vector j lies in a bracket
 #pragma unroll
             for (int j = 0; j < kBatch; ++j) {
-                cm |= in_bracket(q[j].x) ? (1u << (4 * j)) : 0u;
-                cm |= in_bracket(q[j].y) ? (2u << (4 * j)) : 0u;
-                cm |= in_bracket(q[j].z) ? (4u << (4 * j)) : 0u;
-                cm |= in_bracket(q[j].w) ? (8u << (4 * j)) : 0u;
+                if (vmax[j] >= lo_min) {  // a vector whose largest key lies below both brackets holds none of their keys
+                    cm |= in_bracket(q[j].x) ? (1u << (4 * j)) : 0u;
+                    cm |= in_bracket(q[j].y) ? (2u << (4 * j)) : 0u;
+                    cm |= in_bracket(q[j].z) ? (4u << (4 * j)) : 0u;
+                    cm |= in_bracket(q[j].w) ? (8u << (4 * j)) : 0u;
+                }
             }
             if (cm) {  // this lane's keys go to the warp's stage at a position taken from the warp's counter
                 uint32_t pos = atomicAdd(wcount, (uint32_t)__popc(cm));
