@@ -139,3 +139,131 @@ def test_c5b_full_size(B, ora, step, workers):
         assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
     finally:
         B.mlmc_destroy(ctx)
+
+
+# ----------------------------------------------------------------------------------------------
+# the further compressors at the sizes bench.py times them (c3s, c5f, c5r)
+# ----------------------------------------------------------------------------------------------
+def test_c3s_full_size_stopk_many_segments(B, ora):
+    """s-Top-k with L = 1000 segments and a given p on the c3 gradient: every worker's message is one segment of the
+    sorted row (at most s entries); two whole rows go through the oracle, all go through the rank-interval property."""
+    w = wl.C3S
+    torch.cuda.set_device(0)
+    s = w.seg_len
+    L = -(-w.d // s)
+    assert L == 1000
+    p = list(wl.geometric_probs(L))
+    ctx = B.mlmc_create(0, w.d, w.M, 32)
+    try:
+        for step in (0, w.steps - 1):
+            g = wl.gradients(w, step, "cuda")
+            out = B.TopkBuffers(w.M, s)
+            dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+            B.mlmc_compress_stopk(ctx, g, s, p, w.seed, step, out)
+            B.mlmc_aggregate(ctx, B.MLMC_TOPK, out, None, w.M, w.d, dense)
+            assert B.mlmc_get_status(ctx) == B.MLMC_OK
+            level, count, p_sel = out.level.tolist(), out.count.tolist(), out.p_sel.tolist()
+            msgs = []
+            for m in range(w.M):
+                l, n = level[m], count[m]
+                lo, hi = s * l, min(w.d, s * (l + 1))
+                assert 0 <= l < L and n == hi - lo
+                idx = out.idx[m, :n].to(torch.int64) & 0xFFFFFFFF
+                assert bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) < w.d
+                mag = g[m].abs()
+                band = mag[idx]
+                assert int((mag > band.min()).sum()) < hi <= int((mag >= band.min()).sum())
+                assert int((mag > band.max()).sum()) <= lo < int((mag >= band.max()).sum())
+                ref = g[m][idx].double() / p_sel[m]
+                assert bool(((out.val[m, :n].double() - ref).abs() <= VAL_RTOL * ref.abs()).all())
+                msgs.append((out.idx[m, :n].cpu().numpy().view(np.uint32), out.val[m, :n].cpu().numpy()))
+            for m in (1, w.M - 1):
+                o = ora.stopk(wl.as_numpy_bits(g[m:m + 1])[0], s, p, seed=w.seed, step=step, worker=m)
+                if o.margin < MARGIN and level[m] != o.level:
+                    o = ora.stopk(wl.as_numpy_bits(g[m:m + 1])[0], s, p, seed=w.seed, step=step, worker=m, force_level=level[m])
+                assert level[m] == o.level and abs(p_sel[m] - o.p_sel) <= 1e-12 * o.p_sel
+                assert np.array_equal(msgs[m][0], o.idx)
+            ref, scale = ora.aggregate_topk(msgs, w.d)
+            got = dense.cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
+    finally:
+        B.mlmc_destroy(ctx)
+
+
+def test_c5f_full_size_floatbits(B, ora):
+    """Floating-point MLMC on the c5 gradient.  The compressor is element-wise and its probabilities are fixed, so the
+    oracle on a prefix of a row gives that prefix of the message: the first 2^22 coordinates of every worker (exponent
+    bytes, planes, dense mean), and the last, ragged plane words of the row."""
+    w = wl.C5F
+    torch.cuda.set_device(0)
+    mb = list(w.bits)
+    widths = np.diff(np.concatenate([[0], mb]))
+    n_pre = 1 << 22
+    ctx = B.mlmc_create(0, w.d, w.M, 32)
+    try:
+        for step in (0, w.steps - 1):
+            g = wl.gradients(w, step, "cuda")
+            out = B.FloatBuffers(w.M, w.d, int(widths.max()))
+            dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+            B.mlmc_compress_floatbits(ctx, g, mb, None, w.seed, step, out)
+            B.mlmc_aggregate_floatbits(ctx, out, mb, w.M, w.d, dense)
+            assert B.mlmc_get_status(ctx) == B.MLMC_OK
+            level = out.level.tolist()
+            rows = []
+            tail0 = (w.d - 4096) // 32 * 32                     # a word-aligned tail that ends at d
+            for m in range(w.M):
+                wv = int(widths[level[m]])
+                for lo, hi in ((0, n_pre), (tail0, w.d)):
+                    o = ora.floatbits(g[m, lo:hi].cpu().numpy(), mb, None, seed=w.seed, step=step, worker=m,
+                                      force_level=level[m])
+                    assert np.array_equal(out.expo[m, lo:hi].cpu().numpy(), o.expo)
+                    got_planes = out.planes[m, :1 + wv, lo // 32:(hi + 31) // 32].cpu().numpy().view(np.uint32)
+                    assert np.array_equal(got_planes, o.planes)
+                    if lo == 0:
+                        rows.append(o.est)
+                full = ora.floatbits(g[m, :1024].cpu().numpy(), mb, None, seed=w.seed, step=step, worker=m)
+                assert full.margin < MARGIN or full.level == level[m]      # the draw does not depend on the data
+                assert abs(float(out.p_sel[m]) - full.p[level[m]]) <= 1e-15
+            ref, scale = ora.aggregate_dense(rows, n_pre)
+            got = dense[:n_pre].cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
+            assert bool(torch.isfinite(dense).all())
+    finally:
+        B.mlmc_destroy(ctx)
+
+
+def test_c5r_full_size_rtn(B, ora):
+    """Adaptive MLMC-RTN on the c5 gradient: whole rows through the oracle (no sort: a few seconds per row) for two
+    workers, the clipping value of every worker, and the dense mean against the oracle's average of the emitted dense
+    messages on a slice of the coordinates."""
+    w = wl.C5R
+    torch.cuda.set_device(0)
+    r = list(w.bits)
+    ctx = B.mlmc_create(0, w.d, w.M, 32)
+    try:
+        for step, workers in ((0, (0, 5)), (w.steps - 1, (7,))):
+            g = wl.gradients(w, step, "cuda")
+            out = B.RtnBuffers(w.M, w.d)
+            dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+            B.mlmc_compress_rtn(ctx, g, r, None, w.seed, step, out)
+            B.mlmc_aggregate_rtn(ctx, out, w.M, w.d, dense)
+            assert B.mlmc_get_status(ctx) == B.MLMC_OK
+            level, p_sel, c = out.level.tolist(), out.p_sel.tolist(), out.c.cpu().numpy()
+            assert np.array_equal(c, g.abs().max(dim=1).values.cpu().numpy())
+            for m in workers:
+                row = wl.as_numpy_bits(g[m:m + 1])[0]
+                o = ora.rtn(row, r, None, seed=w.seed, step=step, worker=m)
+                if o.margin < MARGIN and level[m] != o.level:
+                    o = ora.rtn(row, r, None, seed=w.seed, step=step, worker=m, force_level=level[m])
+                assert level[m] == o.level and abs(p_sel[m] - o.p_sel) <= 1e-10 * o.p_sel
+                got = out.val[m, :w.d].cpu().numpy().astype(np.float64)
+                assert np.all(np.abs(got - o.val) <= VAL_RTOL * np.abs(o.val) + 1e-45)
+                del got, o, row
+            lo, hi = 40_000_000, 40_000_000 + (1 << 22)
+            rows = [out.val[m, lo:hi].cpu().numpy() for m in range(w.M)]
+            ref, scale = ora.aggregate_dense(rows, hi - lo)
+            got = dense[lo:hi].cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
+            assert bool(torch.isfinite(dense).all())
+    finally:
+        B.mlmc_destroy(ctx)
