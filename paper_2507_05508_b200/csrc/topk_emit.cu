@@ -5,12 +5,13 @@
 // Membership is decided from the two thresholds (Ta, ra), (Tb, rb) of the band; equal-key elements
 // are admitted by their index-ordered rank, so the position of an entry follows from the running counts
 //   C = #{ Tb <= key <= Ta },  A = #{ key == Ta },  B = #{ key == Tb }
-// over the elements before it.  The row is cut into tiles of kEmitTile 32-bit words; only the tiles whose
-// largest key (recorded by the first selection sweep) reaches Tb can hold band entries, the others are never
-// read.  Three kernels, no waiting between thread blocks:
-//   band_count  one warp per listed tile: the tile's C, A, B;
+// over the elements before it.  The row is cut into tiles of kEmitTile 32-bit words, each of kEmitGroups batches;
+// only the batches whose largest key (recorded by the first selection sweep) reaches Tb can hold band entries,
+// the others are never read.  Four kernels, no waiting between thread blocks:
+//   tile_list   one block per worker: the tiles that hold such a batch, each with the mask of those batches;
+//   band_count  one warp per listed tile: the tile's C, A, B over its masked batches;
 //   band_scan   one block per worker: exclusive running totals over the worker's listed tiles;
-//   band_write  one warp per listed tile: reads the tile again and writes its entries at their final positions.
+//   band_write  one warp per listed tile: reads the batches again and writes their entries at their final positions.
 //
 // aggregate: the dense mean (1/M) sum_m g~_m (Alg. 2 "Server aggregates") tiled over the index
 // space; because every message is index-sorted, a tile's entries are one contiguous range per

@@ -6,6 +6,8 @@
 // equal-key elements (in index order) are inside Top-k.  Thresholds come from an MSD radix select
 // on the magnitude key: a 2^15-bin histogram of the leading digit for all queries at once, then two
 // 8-bit digit passes restricted to the boundary bins (fp32 only; a bf16 key is its leading digit).
+// With fixed p the level is drawn first; the boundary bins found by one call are the next call's brackets, so
+// that the first sweep can collect the boundary-bin keys itself.
 #include "common.cuh"
 
 namespace mlmc {
