@@ -53,7 +53,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c5a", "c5b", "c5f", "c5r", "c3s"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c5a", "c5b", "c5f", "c5r", "c3s", "c3a"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -519,7 +519,7 @@ def oracle_sample_step(subs, g_row_np, d_s: int, step: int):
         elif w.kind == "stopk":
             s_len = max(1, min(w.seg_len, d_s))
             L = -(-d_s // s_len)
-            m = oracle.stopk(x, s_len, p=wl.geometric_probs(L), seed=w.seed, step=step, worker=0)
+            m = oracle.stopk(x, s_len, p=None if w.adaptive else wl.geometric_probs(L), seed=w.seed, step=step, worker=0)
             oracle.aggregate_topk([(m.idx, m.val)], d_s)
         elif w.kind == "rtn":
             m = oracle.rtn(x, list(w.bits), p=None, seed=w.seed, step=step, worker=0)

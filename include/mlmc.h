@@ -128,13 +128,17 @@ int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, 
 /* ---- Further multilevel compressors of the paper, same estimator (Eq. 5), same draw, same server average. ---- */
 
 /* s-Top-k (Sec. 2.2 "s-segmented Top-k"; App. D: the segments are those of the sorted vector): level l keeps
- * the l + 1 segments of length s of largest norm, i.e. Top-(s (l + 1)); L = ceil(d / s) levels; the residual of
- * level l is the l-th segment (Sec. 3.2), at most s entries, so capacity >= min(s, d) suffices.
+ * the l + 1 segments of length s of largest norm, i.e. Top-(s (l + 1)); L = ceil(d / s) levels, at most
+ * min(2^20, d_max of the context); the residual of level l is the l-th segment (Sec. 3.2), at most s entries, so
+ * capacity >= min(s, d) suffices.
  *   p  host double[L], all > 0, sum 1 (Alg. 2), or NULL for adaptive p (Lemma 3.4: p^l proportional to the norm of
- *      segment l).  Adaptive p needs every segment norm and is limited to L <= MLMC_MAX_LEVELS; with a given p any
- *      L up to min(2^20, d_max of the context) is accepted, because the level is drawn before the data is read and
- *      only the two thresholds of its segment are selected.
- * Returns MLMC_ERR_ARG when L exceeds those limits. */
+ *      segment l).
+ * Up to MLMC_MAX_LEVELS segments run through mlmc_compress_topk with the schedule k_l = min(d, s (l + 1)).  With more
+ * segments and a given p the level is drawn before the data is read and only the two thresholds of its segment are
+ * selected.  With more segments and adaptive p every segment norm is needed: each row's magnitude keys are sorted
+ * (radix sort), which costs about ten sweeps per row and, at the first such call on a context, one cudaMalloc of
+ * 8 d_max bytes plus a digit table (MLMC_ERR_NOMEM if it fails; freed by mlmc_destroy).
+ * Returns MLMC_ERR_ARG when L exceeds the limit. */
 int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int64_t s,
                         const double* p, uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, void* stream);
 

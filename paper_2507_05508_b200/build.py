@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmlmc.so")
-SOURCES = ["api.cu", "topk_select.cu", "topk_emit.cu", "bitwise.cu", "floatbits.cu", "rtn.cu"]
+SOURCES = ["api.cu", "topk_select.cu", "topk_emit.cu", "bitwise.cu", "floatbits.cu", "rtn.cu", "stopk_sort.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC", "--fmad=true", "-Xptxas", "-v",

@@ -223,6 +223,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_brk = pl.take(sizeof(uint4) * M_max);
     const size_t o_bhit = pl.take(sizeof(int) * M_max);
     const size_t o_bstat = pl.take(sizeof(unsigned long long) * 4);
+    ws.sort_scratch = nullptr;
     ws.sig_d = ws.sig_ld = -1;
     ws.sig_M = ws.sig_L = ws.sig_dtype = -1;
 
@@ -298,6 +299,7 @@ int mlmc_destroy(mlmc_ctx* ctx) {
         delete[] ctx->ws.ev_stop;
         delete[] ctx->ws.ev_id;
     }
+    if (ctx->ws.sort_scratch) cudaFree(ctx->ws.sort_scratch);
     const cudaError_t e = cudaFree(ctx->slab);
     delete ctx;
     return finish(e);
@@ -323,7 +325,8 @@ static const char* const kKernelNames[K_COUNT] = {
     "draw_fixed", "init_queries", "uniforms", "hist1", "resolve1", "sums_candidates", "cand_pass2", "masked_pass2",
     "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
     "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide", "reset",
-    "float_draw", "float_pack", "aggregate_floatbits", "rtn_stats", "rtn_probs_draw", "rtn_emit", "aggregate_dense", "stopk_draw", "stopk_params"};
+    "float_draw", "float_pack", "aggregate_floatbits", "rtn_stats", "rtn_probs_draw", "rtn_emit", "aggregate_dense", "stopk_draw", "stopk_params",
+    "sort_keys", "sort_pass", "segment_norms"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
 
@@ -538,7 +541,27 @@ int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int 
     if (!out || !out->idx || !out->val || !out->count || !out->level || !out->p_sel || out->capacity < 0)
         return MLMC_ERR_ARG;
     Workspace& ws = ctx->ws;
-    if (!p || L > ws.big_cap) return MLMC_ERR_ARG;  // adaptive p needs every segment norm: L <= MLMC_MAX_LEVELS only
+    if (L > ws.big_cap) return MLMC_ERR_ARG;
+    if (!p) {
+        // Adaptive p with many segments (Lemma 3.4 needs the norm of every segment): the rows are sorted, one at a
+        // time, in two key buffers of d_max words that the context allocates at the first such call.
+        DeviceGuard guard(ws.device);
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        if (!ws.sort_scratch) {
+            if (cudaMalloc(&ws.sort_scratch, stopk_sort_scratch_words(ws.d_max) * sizeof(uint32_t)) != cudaSuccess) {
+                cudaGetLastError();
+                ws.sort_scratch = nullptr;
+                return MLMC_ERR_NOMEM;
+            }
+        }
+        cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
+        launch_reset_selection(ws, dtype, d, M, s);
+        launch_hist1(ws, g, dtype, d, M, ld, false, s);  // the batch maxima for the emission, and the NaN / Inf check
+        for (int m = 0; m < M; ++m) launch_stopk_sorted_worker(ws, g, dtype, d, m, ld, s_len, L, seed, step, s);
+        launch_stopk_params(ws, M, s_len, d, out, s);
+        launch_emit(ws, g, dtype, d, M, ld, *out, s);
+        return finish(cudaGetLastError());
+    }
     // normalised p and its running sums in ascending l (the draw is min{ l : u < cdf_l }, the last cdf is 1)
     std::vector<double> pn((size_t)L), cdf((size_t)L);
     double sum = 0.0;

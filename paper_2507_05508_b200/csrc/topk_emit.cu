@@ -26,7 +26,7 @@ namespace {
 
 constexpr int kBandThreads = 256;               // 8 warps per block, one tile per warp at a time
 constexpr int kBatchWords = kEmitRows * 32;     // words a warp holds in registers at a time
-constexpr int kBatches = kEmitTile / kBatchWords;
+static_assert(kEmitTile / kBatchWords == kEmitGroups, "a tile is kEmitGroups batches");
 constexpr int kWriteSlots = 3;                  // shared-memory batches per warp of the write pass
 
 // How a 32-bit word of the gradient row maps to elements: one fp32 element, or two bf16 elements

@@ -62,7 +62,9 @@ C5F = replace(C5A, name="c5f", kind="floatbits", adaptive=False, k_den=0, bits=(
 C5R = replace(C5A, name="c5r", kind="rtn", k_den=0, bits=(2, 4, 8, 16))                                # App. G, adaptive
 C3S = replace(C3, name="c3s", kind="stopk", k_den=0, seg_len=11_690)                                   # App. D, L = 1000, fixed p
 
-ALL = {w.name: w for w in (C1, C2, C3, C4, C5A, C5B, C5F, C5R, C3S)}
+C3A = replace(C3, name="c3a", kind="stopk", adaptive=True, k_den=0, seg_len=116_896)                  # App. D, L = 100, adaptive p
+
+ALL = {w.name: w for w in (C1, C2, C3, C4, C5A, C5B, C5F, C5R, C3S, C3A)}
 
 
 def shrink(w: Workload, d: int, M: Optional[int] = None) -> Workload:

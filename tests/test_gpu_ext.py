@@ -256,12 +256,32 @@ def test_stopk_many_segments_fixed_p(B, ora, ctx, dtype):
         p[l] = 1.0 - 1e-9 * (L - 1)
         check_stopk(B, ora, ctx, g, s, list(p), 3, l, expect_excluded=0)
     out = B.TopkBuffers(3, s)
-    with pytest.raises(B.MlmcError) as e:                                          # adaptive p needs every segment norm
-        B.mlmc_compress_stopk(ctx, g, s, None, 0, 0, out)
-    assert e.value.code == B.MLMC_ERR_ARG
     with pytest.raises(B.MlmcError) as e:
         B.mlmc_compress_stopk(ctx, g, s, [1.0 / L] * (L - 1) + [0.0], 0, 0, out)
     assert e.value.code == B.MLMC_ERR_PROB
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stopk_many_segments_adaptive(B, ora, ctx, dtype):
+    """Adaptive p (Lemma 3.4: p^l proportional to the norm of segment l) with L = 101 and L = 33 segments, the regime of
+    the paper's Adaptive MLMC-Top-k runs (segments of 1 % of the vector and more): every segment norm comes from a
+    sort of the row's magnitude keys."""
+    rng = np.random.default_rng(55)
+    d = 150_001
+    g_np = (rng.standard_normal((3, d)) * 10.0 ** rng.uniform(-3, 0, (3, d))).astype(np.float32)
+    g_np[:, ::7] = np.round(g_np[:, ::7], 3)                                       # ties across segment boundaries
+    g_np[2, 1000:] = 0.0                                                           # a row that is mostly zero: empty tail segments
+    g = to_dev(g_np)
+    if dtype == "bf16":
+        g = padded(g.to(torch.bfloat16), 8)
+    for s, steps in ((1500, 6), (4600, 3)):
+        assert -(-d // s) in (101, 33)
+        for step in range(steps):
+            check_stopk(B, ora, ctx, g, s, None, 23, step, expect_excluded=1)
+    z = to_dev(np.zeros((2, 5000), dtype=np.float32))
+    check_stopk(B, ora, ctx, z, 50, None, 1, 0)                                    # all zero: level 0 with p = 1
+    small = to_dev(rng.standard_normal((2, 70)).astype(np.float32))
+    check_stopk(B, ora, ctx, small, 1, None, 1, 1)                                 # s = 1: Top-k with the unit schedule, L = 70
 
 
 def test_stopk_exponential_decay_closed_forms(B, ora, ctx):
