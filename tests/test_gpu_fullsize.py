@@ -64,6 +64,22 @@ def _topk_fullsize(B, ora, w, step, oracle_workers=(0,)):
                 assert int((mag > hi).sum()) <= kk[l] < int((mag >= hi).sum())
                 del mag, band, ref
             msgs.append((out.idx[m, :n].cpu().numpy().view(np.uint32), out.val[m, :n].cpu().numpy()))
+        if w.adaptive:
+            # Every worker's probabilities and draw, recomputed with library sorts and fp64 sums (neither the CUDA
+            # kernels nor the oracle): p_l = Delta_l / sum Delta from the sorted magnitudes (Lemma 3.4), and the level is
+            # the one the worker's uniform selects, unless the uniform lies within the margin of a cdf boundary.
+            us = B.mlmc_read_u(ctx, w.seed, step, w.M)
+            edges = torch.tensor([0] + list(k), device="cuda")
+            for m in range(w.M):
+                mag2 = g[m].double().abs().sort(descending=True).values.square_()
+                csum = torch.cat([torch.zeros(1, dtype=torch.float64, device="cuda"), mag2.cumsum(0)])
+                delta = (csum[edges[1:]] - csum[edges[:-1]]).clamp_min(0).sqrt()
+                pm = (delta / delta.sum()).cpu().numpy()
+                cdf = np.cumsum(pm)
+                assert abs(p_sel[m] - pm[level[m]]) <= 1e-9 * pm[level[m]]
+                lo_c = cdf[level[m] - 1] if level[m] else 0.0
+                assert lo_c - MARGIN <= us[m] < cdf[level[m]] + MARGIN or level[m] == L - 1
+                del mag2, csum
         for m in oracle_workers:                                         # whole rows through the oracle
             row = wl.as_numpy_bits(g[m:m + 1])[0]
             o = ora.topk(row, k, p=p, seed=w.seed, step=step, worker=m)
