@@ -136,8 +136,9 @@ int mlmc_aggregate(mlmc_ctx* ctx, int kind, const void* msgs, const int32_t* b, 
  * Up to MLMC_MAX_LEVELS segments run through mlmc_compress_topk with the schedule k_l = min(d, s (l + 1)).  With more
  * segments and a given p the level is drawn before the data is read and only the two thresholds of its segment are
  * selected.  With more segments and adaptive p every segment norm is needed: each row's magnitude keys are sorted
- * (radix sort), which costs about ten sweeps per row and, at the first such call on a context, one cudaMalloc of
- * 8 d_max bytes plus a digit table (MLMC_ERR_NOMEM if it fails; freed by mlmc_destroy).
+ * (radix sort, about ten sweeps of the row), as many rows together as fit in 1 GiB of scratch memory (about
+ * 8 d_max + 8 min(2^20, d_max) bytes per row; at least one row), which the first such call on a context takes with
+ * one cudaMalloc (MLMC_ERR_NOMEM if it fails; freed by mlmc_destroy).
  * Returns MLMC_ERR_ARG when L exceeds the limit. */
 int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int M, int64_t ld, int64_t s,
                         const double* p, uint64_t seed, uint64_t step, const mlmc_topk_msgs* out, void* stream);

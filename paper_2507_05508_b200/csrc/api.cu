@@ -153,7 +153,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MLMC_ERR_CUDA;
     if (configure_select_kernels() != MLMC_OK || configure_emit_kernels() != MLMC_OK ||
-        configure_bit_kernels() != MLMC_OK)
+        configure_bit_kernels() != MLMC_OK || configure_sort_kernels() != MLMC_OK)
         return MLMC_ERR_CUDA;
 
     mlmc_ctx* ctx = new (std::nothrow) mlmc_ctx();
@@ -224,6 +224,7 @@ int mlmc_create(mlmc_ctx** out, int device, int64_t d_max, int M_max, int L_max)
     const size_t o_bhit = pl.take(sizeof(int) * M_max);
     const size_t o_bstat = pl.take(sizeof(unsigned long long) * 4);
     ws.sort_scratch = nullptr;
+    ws.sort_rows = 0;
     ws.sig_d = ws.sig_ld = -1;
     ws.sig_M = ws.sig_L = ws.sig_dtype = -1;
 
@@ -326,7 +327,7 @@ static const char* const kKernelNames[K_COUNT] = {
     "resolve2", "cand_pass3", "masked_pass3", "resolve3", "cand_sums", "norm_sweep", "norm_from_hist_bf16", "probs_draw", "copy_probs", "emit", "agg_offsets",
     "aggregate_topk", "absmax", "bit_stats", "bit_probs_draw", "bit_pack", "aggregate_bitwise", "tile_list", "band_count", "band_scan", "bit_pack_wide", "reset",
     "float_draw", "float_pack", "aggregate_floatbits", "rtn_stats", "rtn_probs_draw", "rtn_emit", "aggregate_dense", "stopk_draw", "stopk_params",
-    "sort_keys", "sort_pass", "segment_norms"};
+    "sort_count", "sort_scan", "sort_scatter", "segment_norms"};
 
 int mlmc_kernel_count(void) { return K_COUNT; }
 
@@ -543,12 +544,13 @@ int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int 
     Workspace& ws = ctx->ws;
     if (L > ws.big_cap) return MLMC_ERR_ARG;
     if (!p) {
-        // Adaptive p with many segments (Lemma 3.4 needs the norm of every segment): the rows are sorted, one at a
-        // time, in two key buffers of d_max words that the context allocates at the first such call.
+        // Adaptive p with many segments (Lemma 3.4 needs the norm of every segment): the rows are sorted, several
+        // at a time, in scratch memory that the context allocates at the first such call.
         DeviceGuard guard(ws.device);
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         if (!ws.sort_scratch) {
-            if (cudaMalloc(&ws.sort_scratch, stopk_sort_scratch_words(ws.d_max) * sizeof(uint32_t)) != cudaSuccess) {
+            ws.sort_rows = stopk_sort_rows(ws.d_max, ws.big_cap, ws.M_max);
+            if (cudaMalloc(&ws.sort_scratch, stopk_sort_scratch_bytes(ws.d_max, ws.big_cap, ws.M_max)) != cudaSuccess) {
                 cudaGetLastError();
                 ws.sort_scratch = nullptr;
                 return MLMC_ERR_NOMEM;
@@ -557,7 +559,9 @@ int mlmc_compress_stopk(mlmc_ctx* ctx, const void* g, int dtype, int64_t d, int 
         cudaMemsetAsync(ws.worker_err, 0, sizeof(int) * M, s);
         launch_reset_selection(ws, dtype, d, M, s);
         launch_hist1(ws, g, dtype, d, M, ld, false, s);  // the batch maxima for the emission, and the NaN / Inf check
-        for (int m = 0; m < M; ++m) launch_stopk_sorted_worker(ws, g, dtype, d, m, ld, s_len, L, seed, step, s);
+        for (int m0 = 0; m0 < M; m0 += ws.sort_rows)
+            launch_stopk_sorted_rows(ws, g, dtype, d, m0, (M - m0 < ws.sort_rows) ? M - m0 : ws.sort_rows, ld, s_len, L,
+                                     seed, step, s);
         launch_stopk_params(ws, M, s_len, d, out, s);
         launch_emit(ws, g, dtype, d, M, ld, *out, s);
         return finish(cudaGetLastError());

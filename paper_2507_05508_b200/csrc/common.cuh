@@ -56,7 +56,7 @@ enum KernelId {
     K_MASKED3, K_RESOLVE3, K_CAND_SUMS, K_NORM_SWEEP, K_NORM_HIST, K_PROBS_DRAW, K_COPY_PROBS, K_EMIT, K_AGG_OFFSETS, K_AGG_TOPK,
     K_ABSMAX, K_BIT_STATS, K_BIT_DRAW, K_BIT_PACK, K_AGG_BIT, K_TILE_LIST, K_BAND_COUNT, K_BAND_SCAN, K_BIT_PACK_WIDE, K_RESET,
     K_FLOAT_DRAW, K_FLOAT_PACK, K_AGG_FLOAT, K_RTN_STATS, K_RTN_DRAW, K_RTN_EMIT, K_AGG_DENSE, K_STOPK_DRAW, K_STOPK_PARAMS,
-    K_SORT_KEYS, K_SORT_PASS, K_SEG_NORMS, K_COUNT
+    K_SORT_COUNT, K_SORT_SCAN, K_SORT_SCATTER, K_SEG_NORMS, K_COUNT
 };
 
 constexpr int kTimingPool = 2048;  // event pairs kept between two reads
@@ -124,7 +124,8 @@ struct Workspace {
     double* p_big;               // [big_cap]
     double* cdf_big;             // [big_cap]
     int64_t big_cap;
-    uint32_t* sort_scratch;      // two key buffers of d_max words and the digit table of the radix sort; allocated at first use
+    uint32_t* sort_scratch;      // key buffers, digit tables and segment norms of the radix sort, for sort_rows rows; allocated at first use
+    int sort_rows;               // rows that are sorted together
     // RTN: per-block residual energies of every level
     double* rtn_partial;         // [M][rtn_ctas][kMaxLevels]
     int rtn_ctas, cur_rtn_ctas;
@@ -327,8 +328,10 @@ void launch_stopk_draw(Workspace& ws, int M, int64_t L, int64_t s_len, int64_t d
                        cudaStream_t s);
 void launch_stopk_params(Workspace& ws, int M, int64_t s_len, int64_t d, const mlmc_topk_msgs* out, cudaStream_t s);
 // stopk_sort.cu: s-Top-k with adaptive p and many segments
-size_t stopk_sort_scratch_words(int64_t d_max);
-void launch_stopk_sorted_worker(Workspace& ws, const void* g, int dtype, int64_t d, int m, int64_t ld, int64_t s_len,
-                                int64_t L, uint64_t seed, uint64_t step, cudaStream_t s);
+int configure_sort_kernels();
+int stopk_sort_rows(int64_t d_max, int64_t big_cap, int M_max);
+size_t stopk_sort_scratch_bytes(int64_t d_max, int64_t big_cap, int M_max);
+void launch_stopk_sorted_rows(Workspace& ws, const void* g, int dtype, int64_t d, int m0, int rows, int64_t ld,
+                              int64_t s_len, int64_t L, uint64_t seed, uint64_t step, cudaStream_t s);
 
 }  // namespace mlmc

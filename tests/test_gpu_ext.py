@@ -284,6 +284,20 @@ def test_stopk_many_segments_adaptive(B, ora, ctx, dtype):
     check_stopk(B, ora, ctx, small, 1, None, 1, 1)                                 # s = 1: Top-k with the unit schedule, L = 70
 
 
+def test_stopk_adaptive_rows_sorted_in_groups(B, ora):
+    """A context whose rows are too long to be sorted all together (the scratch memory of the sort holds two of its
+    three rows): the second group reuses the buffers of the first."""
+    rng = np.random.default_rng(57)
+    d = 60_011
+    g = to_dev((rng.standard_normal((3, d)) * 10.0 ** rng.uniform(-3, 0, (3, d))).astype(np.float32))
+    big = B.mlmc_create(0, 48_000_000, 3, 32)
+    try:
+        for step in range(3):
+            check_stopk(B, ora, big, g, 601, None, 29, step, expect_excluded=1)   # L = 100
+    finally:
+        B.mlmc_destroy(big)
+
+
 def test_stopk_exponential_decay_closed_forms(B, ora, ctx):
     """Assumption 3.5 / Lemma 3.6 on the device: |v(j)| = a exp(-r j / 2) on the sorted vector, s L = d with L = 32
     segments; the residual norms of mlmc_level_probs follow the closed form of App. E, and the adaptive second moment

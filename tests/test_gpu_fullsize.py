@@ -206,6 +206,62 @@ def test_c3s_full_size_stopk_many_segments(B, ora):
         B.mlmc_destroy(ctx)
 
 
+def test_c3a_full_size_stopk_adaptive_many_segments(B, ora):
+    """s-Top-k with L = 100 segments and adaptive p (Lemma 3.4) on the c3 gradient, the sorted path at the size
+    bench.py times it (the 16 rows are sorted in two groups).  Every worker: the band is the rank interval of its
+    segment, and p_sel and the draw agree with segment norms recomputed by library sorts and fp64 sums; two whole rows
+    go through the oracle."""
+    w = wl.C3A
+    torch.cuda.set_device(0)
+    s = w.seg_len
+    L = -(-w.d // s)
+    assert L == 100 and w.adaptive
+    ctx = B.mlmc_create(0, w.d, w.M, 32)
+    try:
+        for step in (0, w.steps - 1):
+            g = wl.gradients(w, step, "cuda")
+            out = B.TopkBuffers(w.M, s)
+            dense = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+            B.mlmc_compress_stopk(ctx, g, s, None, w.seed, step, out)
+            B.mlmc_aggregate(ctx, B.MLMC_TOPK, out, None, w.M, w.d, dense)
+            assert B.mlmc_get_status(ctx) == B.MLMC_OK
+            level, count, p_sel = out.level.tolist(), out.count.tolist(), out.p_sel.tolist()
+            us = B.mlmc_read_u(ctx, w.seed, step, w.M)
+            edges = torch.arange(0, L + 1, device="cuda").mul_(s).clamp_(max=w.d)
+            msgs = []
+            for m in range(w.M):
+                l, n = level[m], count[m]
+                lo, hi = s * l, min(w.d, s * (l + 1))
+                assert 0 <= l < L and n == hi - lo
+                idx = out.idx[m, :n].to(torch.int64) & 0xFFFFFFFF
+                assert bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) < w.d
+                mag = g[m].abs()
+                band = mag[idx]
+                assert int((mag > band.min()).sum()) < hi <= int((mag >= band.min()).sum())
+                assert int((mag > band.max()).sum()) <= lo < int((mag >= band.max()).sum())
+                mag2 = mag.double().sort(descending=True).values.square_()
+                csum = torch.cat([torch.zeros(1, dtype=torch.float64, device="cuda"), mag2.cumsum(0)])
+                delta = (csum[edges[1:]] - csum[edges[:-1]]).clamp_min(0).sqrt()
+                pm = (delta / delta.sum()).cpu().numpy()
+                cdf = np.cumsum(pm)
+                assert abs(p_sel[m] - pm[l]) <= 1e-9 * pm[l]
+                assert ((cdf[l - 1] if l else 0.0) - MARGIN <= us[m] < cdf[l] + MARGIN) or l == L - 1
+                ref = g[m][idx].double() / p_sel[m]
+                assert bool(((out.val[m, :n].double() - ref).abs() <= VAL_RTOL * ref.abs()).all())
+                msgs.append((out.idx[m, :n].cpu().numpy().view(np.uint32), out.val[m, :n].cpu().numpy()))
+            for m in (0, w.M - 1):                                       # one row of each group
+                o = ora.stopk(wl.as_numpy_bits(g[m:m + 1])[0], s, None, seed=w.seed, step=step, worker=m)
+                if o.margin < MARGIN and level[m] != o.level:
+                    o = ora.stopk(wl.as_numpy_bits(g[m:m + 1])[0], s, None, seed=w.seed, step=step, worker=m, force_level=level[m])
+                assert level[m] == o.level and abs(p_sel[m] - o.p_sel) <= 1e-11 * o.p_sel
+                assert np.array_equal(msgs[m][0], o.idx)
+            ref, scale = ora.aggregate_topk(msgs, w.d)
+            got = dense.cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(got - ref) <= AGG_RTOL * scale + 1e-45)
+    finally:
+        B.mlmc_destroy(ctx)
+
+
 def test_c5f_full_size_floatbits(B, ora):
     """Floating-point MLMC on the c5 gradient.  The compressor is element-wise and its probabilities are fixed, so the
     oracle on a prefix of a row gives that prefix of the message: the first 2^22 coordinates of every worker (exponent
