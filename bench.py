@@ -15,6 +15,7 @@ Prints ONE JSON line on rank 0.
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import subprocess
@@ -124,7 +125,7 @@ def max_over_ranks(local_ms: float, world: int, device: str) -> float:
 # clocks
 # --------------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -133,12 +134,22 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(device_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def _stamp(text: str):
+        try:
+            return datetime.datetime.strptime(text.strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except Exception:
+            return None
+
+    def stop(self, t0: float = None, t1: float = None):
+        """Median SM clock, reasons and power over the samples taken between the wall-clock times t0 and t1 (the
+        timed region; the sampler is started before the warm-up so that it is already running); all samples when
+        none carries a usable time stamp inside the window."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -152,14 +163,18 @@ class ClockSampler:
         rows = [r.strip().split(",") for r in self.tmp.read().splitlines() if r.strip()]
         self.tmp.close()
         os.unlink(self.tmp.name)
+        if t0 is not None and t1 is not None:
+            inside = [r for r in rows if (lambda ts: ts is not None and t0 <= ts <= t1)(self._stamp(r[0]))]
+            if inside:
+                rows = inside
         sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             try:
-                sm.append(float(r[0]))
-                mx.append(float(r[1]))
-                power.append(float(r[2]))
-                for name, v in zip(names, r[3:7]):
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+                power.append(float(r[3]))
+                for name, v in zip(names, r[4:8]):
                     if v.strip().lower().startswith("active"):
                         reasons.add(name)
             except Exception:
@@ -314,6 +329,7 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
     small = sweep_bytes <= 126e6
     flush = torch.empty(int(252e6) // 4, dtype=torch.float32, device=r.dev) if small else None
 
+    sampler = ClockSampler(local)  # running before the warm-up; only its samples inside the timed region are kept
     for i in range(max(warmup, 3)):
         r.step(i)
     torch.cuda.synchronize()
@@ -321,7 +337,6 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
 
     # ---- headline loop: exactly `steps` steps, device-timed, per-kernel timing off
     launches0 = B.mlmc_launch_count(r.ctx)
-    sampler = ClockSampler(local)
     barrier(world)
     torch.cuda.synchronize()
     t_wall0 = time.time()
@@ -345,7 +360,7 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
         local_ms = e0.elapsed_time(e1)
     barrier(world)
     t_wall = time.time() - t_wall0
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_wall0, t_wall0 + t_wall)
     total_ms = max_over_ranks(local_ms, world, r.dev)
     launches = B.mlmc_launch_count(r.ctx) - launches0
     status = B.mlmc_get_status(r.ctx)
