@@ -57,7 +57,7 @@ C5A = Workload("c5a", "topk", 124_439_808, 8, "f32", True, 4, 10, "normal", "seg
                outlier_frac=1e-3, outlier_mult=100.0, k_den=10000)
 C5B = replace(C5A, name="c5b", kind="bitwise", k_den=0, bits=(1, 2, 4, 8, 16, 23))
 
-# The further compressors of the paper on the same synthetic gradients (not BASELINE configs: measured beside them).
+# The further compressors of the paper on the same synthetic gradients (not among the five benchmark configurations: measured beside them).
 C5F = replace(C5A, name="c5f", kind="floatbits", adaptive=False, k_den=0, bits=(1, 2, 4, 8, 16, 23))   # App. B, fixed p
 C5R = replace(C5A, name="c5r", kind="rtn", k_den=0, bits=(2, 4, 8, 16))                                # App. G, adaptive
 C3S = replace(C3, name="c3s", kind="stopk", k_den=0, seg_len=11_690)                                   # App. D, L = 1000, fixed p
