@@ -306,6 +306,15 @@ def kernel_alg_bytes(name: str, sweep: float, msg: dict, dense: float, read_frac
     return table.get(name)
 
 
+def sort_step_bytes(name: str, sweep: float, elem: int):
+    """Bytes per STEP of the radix-sort kernels of the adaptive s-Top-k path with many segments (their launches
+    differ in size: the rows are sorted in groups): 32-bit keys, 4 passes for fp32 and 2 for bf16, the first pass
+    reading the gradient itself; a count pass reads its input, a scatter pass reads it and writes the keys."""
+    keys, passes = sweep * 4.0 / elem, (4 if elem == 4 else 2)
+    reads = sweep + (passes - 1) * keys
+    return {"sort_count": reads, "sort_scatter": reads + passes * keys, "segment_norms": keys}.get(name)
+
+
 def l2_policy(sweep_bytes: float, n_batches: int) -> str:
     l2 = 126e6
     if sweep_bytes > l2:
@@ -400,6 +409,9 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
         kb = kernel_alg_bytes(name, sweep_bytes, msg_by_kind, dense_bytes, emit_read_frac, adaptive_topk)
         avg_ms = ms / n
         ach = None if not kb else kb / (avg_ms * 1e-3) / 1e9
+        sb = sort_step_bytes(name, sweep_bytes, elem_size(w))
+        if sb:
+            ach = sb / (ms / probe * 1e-3) / 1e9
         kernels[name] = {"ms_per_step": round(ms / probe, 4), "launches_per_step": n / probe,
                          "share": round(ms / t_all, 4), "achieved_gbs": None if ach is None else round(ach, 1),
                          "frac": None if ach is None else round(ach / peak, 4)}
