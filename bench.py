@@ -56,7 +56,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "c5a", "c5b", "c5f", "c5r", "c3s", "c3a"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true", help="skip the shorter runs of c4, c5a, c5b and c3 reported under `also`")
     ap.add_argument("--also-steps", type=int, default=10)
@@ -190,7 +190,10 @@ class ClockSampler:
 # the CUDA arm
 # --------------------------------------------------------------------------------------------------
 class Runner:
-    """Owns the buffers of one workload (one or two variants over the same batch) and runs steps through the C ABI."""
+    """Owns the buffers of one workload (one or two variants over the same batch) and runs steps through the C ABI.
+    Every variant has its own context, message buffers and dense output; the variants of a step do not depend on one
+    another, so a step runs them side by side, each on a CUDA stream of its own (a context serves one stream at a
+    time), forked from and joined to the stream that times the step."""
 
     def __init__(self, subs, device_index: int, n_batches: int = 2, rank: int = 0):
         import torch
@@ -200,11 +203,12 @@ class Runner:
         w = self.w = subs[0]
         self.dev = f"cuda:{device_index}"
         torch.cuda.set_device(device_index)
-        self.ctx = B.mlmc_create(device_index, w.d, w.M, 32)
+        self.ctxs = [B.mlmc_create(device_index, w.d, w.M, 32) for _ in subs]
+        self.side = [None] + [torch.cuda.Stream(device=self.dev) for _ in subs[1:]]
         sc = wl.scales(w, self.dev)
         self.batches = [wl.gradients(w, 1000 * rank + i, self.dev, sc) for i in range(n_batches)]
         del sc
-        self.dense = torch.empty(w.d, dtype=torch.float32, device=self.dev)
+        self.denses = [torch.empty(w.d, dtype=torch.float32, device=self.dev) for _ in subs]
         self.plan = []
         for x in subs:
             if x.kind == "topk":
@@ -229,25 +233,76 @@ class Runner:
         self.L = [len(pl[1]) for pl in self.plan]
         torch.cuda.synchronize()
 
-    def step(self, i: int, g=None):
+    def _variant(self, j: int, i: int, g):
         B = self.B
+        ctx, dense = self.ctxs[j], self.denses[j]
+        x, sched, p, msgs = self.plan[j]
+        if x.kind == "topk":
+            B.mlmc_compress_topk(ctx, g, sched, p, x.seed, i, msgs)
+            B.mlmc_aggregate(ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, dense)
+        elif x.kind == "stopk":
+            B.mlmc_compress_stopk(ctx, g, x.seg_len, p, x.seed, i, msgs)
+            B.mlmc_aggregate(ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, dense)
+        elif x.kind == "rtn":
+            B.mlmc_compress_rtn(ctx, g, sched[:-1], p, x.seed, i, msgs)
+            B.mlmc_aggregate_rtn(ctx, msgs, x.M, x.d, dense)
+        elif x.kind == "floatbits":
+            B.mlmc_compress_floatbits(ctx, g, sched, p, x.seed, i, msgs)
+            B.mlmc_aggregate_floatbits(ctx, msgs, sched, x.M, x.d, dense)
+        else:
+            B.mlmc_compress_bitwise(ctx, g, sched, p, x.seed, i, msgs)
+            B.mlmc_aggregate(ctx, B.MLMC_BITWISE, msgs, sched, x.M, x.d, dense)
+
+    def step(self, i: int, g=None, side_by_side: bool = True):
+        torch = self.torch
         g = self.batches[i % len(self.batches)] if g is None else g
-        for x, sched, p, msgs in self.plan:
-            if x.kind == "topk":
-                B.mlmc_compress_topk(self.ctx, g, sched, p, x.seed, i, msgs)
-                B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, self.dense)
-            elif x.kind == "stopk":
-                B.mlmc_compress_stopk(self.ctx, g, x.seg_len, p, x.seed, i, msgs)
-                B.mlmc_aggregate(self.ctx, B.MLMC_TOPK, msgs, None, x.M, x.d, self.dense)
-            elif x.kind == "rtn":
-                B.mlmc_compress_rtn(self.ctx, g, sched[:-1], p, x.seed, i, msgs)
-                B.mlmc_aggregate_rtn(self.ctx, msgs, x.M, x.d, self.dense)
-            elif x.kind == "floatbits":
-                B.mlmc_compress_floatbits(self.ctx, g, sched, p, x.seed, i, msgs)
-                B.mlmc_aggregate_floatbits(self.ctx, msgs, sched, x.M, x.d, self.dense)
-            else:
-                B.mlmc_compress_bitwise(self.ctx, g, sched, p, x.seed, i, msgs)
-                B.mlmc_aggregate(self.ctx, B.MLMC_BITWISE, msgs, sched, x.M, x.d, self.dense)
+        if len(self.plan) == 1 or not side_by_side:
+            for j in range(len(self.plan)):
+                self._variant(j, i, g)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        joins = []
+        for j in range(1, len(self.plan)):
+            self.side[j].wait_event(fork)          # the batch is ready
+            with torch.cuda.stream(self.side[j]):
+                self._variant(j, i, g)
+                done = torch.cuda.Event()
+                done.record(self.side[j])
+            joins.append(done)
+        self._variant(0, i, g)
+        for done in joins:
+            main.wait_event(done)                  # the step ends when every variant has
+
+    def status(self) -> int:
+        for ctx in self.ctxs:
+            st = self.B.mlmc_get_status(ctx)
+            if st != 0:
+                return st
+        return 0
+
+    def launch_count(self) -> int:
+        return sum(self.B.mlmc_launch_count(ctx) for ctx in self.ctxs)
+
+    def timing_enable(self, on: bool):
+        for ctx in self.ctxs:
+            self.B.mlmc_timing_enable(ctx, on)
+
+    def timing_read(self) -> dict:
+        out = {}
+        for ctx in self.ctxs:
+            for name, (ms, n) in self.B.mlmc_timing_read(ctx).items():
+                a = out.setdefault(name, [0.0, 0])
+                a[0] += ms
+                a[1] += n
+        return {k: (v[0], v[1]) for k, v in out.items()}
+
+    def topk_ctx(self):
+        for ctx, (x, _, _, _) in zip(self.ctxs, self.plan):
+            if x.kind in ("topk", "stopk"):
+                return ctx
+        return None
 
     def message_bytes(self):
         """Per variant kind: bytes of the messages of the last step (written once by compress, read once by aggregate)."""
@@ -266,7 +321,8 @@ class Runner:
         return out
 
     def close(self):
-        self.B.mlmc_destroy(self.ctx)
+        for ctx in self.ctxs:
+            self.B.mlmc_destroy(ctx)
 
 
 def sweeps_charged(w, emit_read_frac=None) -> float:
@@ -342,10 +398,10 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
     for i in range(max(warmup, 3)):
         r.step(i)
     torch.cuda.synchronize()
-    assert B.mlmc_get_status(r.ctx) == 0, "device status after warm-up"
+    assert r.status() == 0, "device status after warm-up"
 
     # ---- headline loop: exactly `steps` steps, device-timed, per-kernel timing off
-    launches0 = B.mlmc_launch_count(r.ctx)
+    launches0 = r.launch_count()
     barrier(world)
     torch.cuda.synchronize()
     t_wall0 = time.time()
@@ -371,31 +427,31 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
     t_wall = time.time() - t_wall0
     clocks = sampler.stop(t_wall0, t_wall0 + t_wall)
     total_ms = max_over_ranks(local_ms, world, r.dev)
-    launches = B.mlmc_launch_count(r.ctx) - launches0
-    status = B.mlmc_get_status(r.ctx)
+    launches = r.launch_count() - launches0
+    status = r.status()
     ms_per_step = total_ms / steps
     value = world * len(subs) * sweep_bytes / (ms_per_step * 1e-3) / 1e9
 
     # ---- second loop, same steps: per-kernel event pairs, message volume, listed tiles (read back after every step)
-    B.mlmc_timing_enable(r.ctx, True)
+    r.timing_enable(True)
     per_kernel, msg_acc = {}, {}
     listed_acc, listed_n = 0.0, 0
     probe = min(steps, 16)
     for i in range(probe):
         if small:
             flush.fill_(float(i))
-        r.step(warmup + i)
-        for name, (ms, n) in B.mlmc_timing_read(r.ctx).items():
+        r.step(warmup + i, side_by_side=False)  # one variant after the other: the event pairs time kernels that run alone
+        for name, (ms, n) in r.timing_read().items():
             acc = per_kernel.setdefault(name, [0.0, 0])
             acc[0] += ms
             acc[1] += n
         for kind, v in r.message_bytes().items():
             msg_acc[kind] = msg_acc.get(kind, 0.0) + v
         if any(x.kind in ("topk", "stopk") for x in subs):
-            listed, tiles = B.mlmc_read_listed_tiles(r.ctx, w.M)
+            listed, tiles = B.mlmc_read_listed_tiles(r.topk_ctx(), w.M)
             listed_acc += sum(listed) / float(max(1, tiles * w.M))
             listed_n += 1
-    B.mlmc_timing_enable(r.ctx, False)
+    r.timing_enable(False)
     emit_read_frac = (listed_acc / listed_n) if listed_n else None
     msg_by_kind = {kind: v / probe for kind, v in msg_acc.items()}
     msg_bytes = sum(msg_by_kind.values())
@@ -434,33 +490,60 @@ def measure(subs, local: int, rank: int, world: int, steps: int, warmup: int, pe
     if e2e_steps > 0:
         host_in = torch.empty(r.batches[0].shape, dtype=r.batches[0].dtype, pin_memory=True)
         host_in.copy_(r.batches[0])
-        host_out = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
-        g_dev = r.batches[1 % len(r.batches)]
+        host_out = [torch.empty(w.d, dtype=torch.float32, pin_memory=True) for _ in r.denses]  # every variant's mean
+        # Three streams, as a training loop would run it: the copy of step i + 1's gradients into the other device
+        # batch and the read-back of step i's means run beside the compute of the steps between them.  Every step
+        # copies its whole input from pinned host memory and reads every variant's dense mean back; the timed region
+        # starts before the first copy and ends after the last read-back.
+        bufs = r.batches[:2] if len(r.batches) >= 2 else [r.batches[0], torch.empty_like(r.batches[0])]
+        s_in, s_out = torch.cuda.Stream(device=r.dev), torch.cuda.Stream(device=r.dev)
+        main = torch.cuda.current_stream()
 
-        def e2e_step(i):
-            g_dev.copy_(host_in, non_blocking=True)
-            r.step(i, g_dev)
-            host_out.copy_(r.dense, non_blocking=True)
+        def e2e_run(n, first):
+            computed, copied_out = {}, None
+            for k in range(n):
+                i = first + k
+                buf = bufs[k % 2]
+                if k >= 2:
+                    s_in.wait_event(computed[k - 2])       # the step that read this batch has finished
+                with torch.cuda.stream(s_in):
+                    buf.copy_(host_in, non_blocking=True)
+                    arrived = torch.cuda.Event()
+                    arrived.record(s_in)
+                main.wait_event(arrived)
+                if copied_out is not None:
+                    main.wait_event(copied_out)            # the means of the step before are on the host
+                r.step(i, buf)
+                computed[k] = torch.cuda.Event()
+                computed[k].record(main)
+                s_out.wait_event(computed[k])
+                with torch.cuda.stream(s_out):
+                    for dst, src in zip(host_out, r.denses):
+                        dst.copy_(src, non_blocking=True)
+                    copied_out = torch.cuda.Event()
+                    copied_out.record(s_out)
+            main.wait_event(copied_out)
 
-        e2e_step(0)
+        e2e_run(1, 0)
         torch.cuda.synchronize()
         barrier(world)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for i in range(e2e_steps):
-            e2e_step(i + 1)
+        s_in.wait_event(a)
+        e2e_run(e2e_steps, 1)
         b.record()
         torch.cuda.synchronize()
         barrier(world)
         e2e_ms = max_over_ranks(a.elapsed_time(b), world, r.dev) / e2e_steps
         e2e = {"value": round(world * len(subs) * sweep_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
-               "h2d_bytes_per_step": int(sweep_bytes), "d2h_bytes_per_step": int(dense_bytes),
+               "h2d_bytes_per_step": int(sweep_bytes), "d2h_bytes_per_step": int(dense_bytes) * len(r.denses),
                "ms_per_step": round(e2e_ms, 3)}
         del host_in, host_out
 
     words = describe(subs) + f", L={r.L}"
     if len(subs) > 1:
-        words += f"; value counts the gradient bytes once per variant ({len(subs)} x M*d*4 per step)"
+        words += (f"; value counts the gradient bytes once per variant ({len(subs)} x M*d*4 per step); the variants of "
+                  f"a step run side by side on {len(subs)} CUDA streams, a context each")
     res = {
         "value": round(value, 2), "ms_per_step": round(ms_per_step, 4), "steps": steps,
         "config": {"workload": words, "l2_policy": l2_policy(sweep_bytes, len(r.batches)),
