@@ -204,7 +204,9 @@ class Runner:
         self.dev = f"cuda:{device_index}"
         torch.cuda.set_device(device_index)
         self.ctxs = [B.mlmc_create(device_index, w.d, w.M, 32) for _ in subs]
-        self.side = [None] + [torch.cuda.Stream(device=self.dev) for _ in subs[1:]]
+        # the last variant runs on the timing stream, the ones before it on high-priority streams (the Top-k pipeline,
+        # listed first, is a chain of many short kernels that should not queue behind the other variant's sweeps)
+        self.side = [torch.cuda.Stream(device=self.dev, priority=-1) for _ in subs[:-1]] + [None]
         sc = wl.scales(w, self.dev)
         self.batches = [wl.gradients(w, 1000 * rank + i, self.dev, sc) for i in range(n_batches)]
         del sc
@@ -264,14 +266,14 @@ class Runner:
         fork = torch.cuda.Event()
         fork.record(main)
         joins = []
-        for j in range(1, len(self.plan)):
+        for j in range(len(self.plan) - 1):
             self.side[j].wait_event(fork)          # the batch is ready
             with torch.cuda.stream(self.side[j]):
                 self._variant(j, i, g)
                 done = torch.cuda.Event()
                 done.record(self.side[j])
             joins.append(done)
-        self._variant(0, i, g)
+        self._variant(len(self.plan) - 1, i, g)
         for done in joins:
             main.wait_event(done)                  # the step ends when every variant has
 
