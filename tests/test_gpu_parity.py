@@ -481,3 +481,56 @@ def test_run_to_run_determinism(B, ctx):
             assert all(torch.equal(a, b) for a, b in zip(snap[2], ref[2]))
             assert all(torch.equal(a, b) for a, b in zip(snap[3], ref[3]))
         ref = snap
+
+
+def test_two_contexts_side_by_side_on_two_streams(B, ctx):
+    """A context serves one stream at a time; two contexts share nothing.  The Top-k and the bit-wise pipeline of a
+    step, run side by side on two streams with a context each (as bench.py runs its two-variant workload), give
+    bit for bit what they give one after the other on one stream (which the tests above compare with the oracle)."""
+    w = wl.shrink(wl.C5A, 1_500_003, 4)
+    k = wl.topk_schedule(w)
+    bits = list(wl.C5B.bits)
+    widths = [bits[0]] + [bits[i] - bits[i - 1] for i in range(1, len(bits))]
+    sc = wl.scales(w, "cuda")
+    other = B.mlmc_create(0, w.d, w.M, 32)
+    side = torch.cuda.Stream(priority=-1)
+    try:
+        for step in range(4):
+            g = padded(wl.gradients(w, step, "cuda", sc), 4)
+
+            def run(side_by_side):
+                mt, mb = B.TopkBuffers(w.M, wl.max_band(k)), B.BitBuffers(w.M, w.d, max(widths))
+                dt = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+                db = torch.full((w.d,), float("nan"), dtype=torch.float32, device="cuda")
+                main = torch.cuda.current_stream()
+                if side_by_side:
+                    fork = torch.cuda.Event()
+                    fork.record(main)
+                    side.wait_event(fork)
+                    with torch.cuda.stream(side):
+                        B.mlmc_compress_topk(other, g, k, None, w.seed, step, mt)
+                        B.mlmc_aggregate(other, B.MLMC_TOPK, mt, None, w.M, w.d, dt)
+                        done = torch.cuda.Event()
+                        done.record(side)
+                    B.mlmc_compress_bitwise(ctx, g, bits, None, w.seed, step, mb)
+                    B.mlmc_aggregate(ctx, B.MLMC_BITWISE, mb, bits, w.M, w.d, db)
+                    main.wait_event(done)
+                else:
+                    B.mlmc_compress_topk(ctx, g, k, None, w.seed, step, mt)
+                    B.mlmc_aggregate(ctx, B.MLMC_TOPK, mt, None, w.M, w.d, dt)
+                    B.mlmc_compress_bitwise(ctx, g, bits, None, w.seed, step, mb)
+                    B.mlmc_aggregate(ctx, B.MLMC_BITWISE, mb, bits, w.M, w.d, db)
+                torch.cuda.synchronize()
+                assert B.mlmc_get_status(ctx) == 0 and B.mlmc_get_status(other) == 0
+                n = mt.count.tolist()
+                return (mt.level.tolist(), mt.p_sel.tolist(), n, [mt.idx[m, :n[m]].clone() for m in range(w.M)],
+                        [mt.val[m, :n[m]].clone() for m in range(w.M)], dt, mb.level.tolist(), mb.p_sel.tolist(),
+                        mb.gmax.clone(), [mb.planes[m, :1 + widths[l]].clone() for m, l in enumerate(mb.level.tolist())], db)
+
+            a, b = run(False), run(True)
+            assert a[0] == b[0] and a[1] == b[1] and a[2] == b[2] and a[6] == b[6] and a[7] == b[7]
+            assert all(torch.equal(x, y) for x, y in zip(a[3], b[3])) and all(torch.equal(x, y) for x, y in zip(a[4], b[4]))
+            assert torch.equal(a[5], b[5]) and torch.equal(a[8], b[8]) and torch.equal(a[10], b[10])
+            assert all(torch.equal(x, y) for x, y in zip(a[9], b[9]))
+    finally:
+        B.mlmc_destroy(other)
