@@ -27,7 +27,7 @@
  *    rounds, u = (h >> 11) * 2^-53; cdf accumulated in ascending l in fp64, the cdf of the last level
  *    with p > 0 set to 1, l* = min{ l : u < cdf_l }.
  *  - One mlmc_ctx serves one stream at a time.  Contexts share nothing: calls on different contexts may run
- *    side by side on different streams (and from different host threads).
+ *    side by side on different streams.
  */
 #ifndef MLMC_H
 #define MLMC_H
