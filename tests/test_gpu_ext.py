@@ -284,6 +284,20 @@ def test_stopk_many_segments_adaptive(B, ora, ctx, dtype):
     check_stopk(B, ora, ctx, small, 1, None, 1, 1)                                 # s = 1: Top-k with the unit schedule, L = 70
 
 
+@pytest.mark.parametrize("d,s", [(8192, 100), (8193, 100), (16384, 37), (131_077, 1), (40_000, 1023), (40_000, 1024), (200_000, 4096), (200_000, 4097)])
+def test_stopk_adaptive_sort_edges(B, ora, ctx, d, s):
+    """The sorted path at the edges of its tiling: rows of exactly one and two sort tiles and one key more, one
+    entry per segment (L = d), and segment lengths on both sides of the switch between a warp and a block per
+    segment and of the chunk length of the norms."""
+    rng = np.random.default_rng(59 + d + s)
+    g_np = (rng.standard_normal((2, d)) * 10.0 ** rng.uniform(-2, 0, (2, d))).astype(np.float32)
+    g_np[:, ::5] = np.round(g_np[:, ::5], 2)                                       # ties
+    g = to_dev(g_np)
+    assert -(-d // s) > 32
+    for step in range(2):
+        check_stopk(B, ora, ctx, g, s, None, 31, step, expect_excluded=1)
+
+
 def test_stopk_adaptive_rows_sorted_in_groups(B, ora):
     """A context whose rows are too long to be sorted all together (the scratch memory of the sort holds two of its
     three rows): the second group reuses the buffers of the first."""
